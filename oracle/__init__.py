@@ -51,26 +51,29 @@ class Adam:
                      int(self.drop_eps_term), int(self.identity))
 
 
+def _bind(lib):
+    fp, dp, ip = C.POINTER(C.c_float), C.POINTER(C.c_double), C.POINTER(C.c_int32)
+    ap = C.POINTER(_Adam)
+    lib.sama_oracle_adapt.argtypes = [C.c_int64, fp, fp, fp, fp, ap, dp]
+    lib.sama_oracle_adapt.restype = None
+    lib.sama_oracle_sumsq.argtypes = [C.c_int64, dp]
+    lib.sama_oracle_sumsq.restype = C.c_double
+    lib.sama_oracle_perturb.argtypes = [C.c_int64, fp, dp, C.c_double, dp, dp, dp]
+    lib.sama_oracle_perturb.restype = C.c_int
+    lib.sama_oracle_losses.argtypes = [C.c_int32, ip, dp, fp, ip, C.c_int32, dp, dp]
+    lib.sama_oracle_losses.restype = None
+    lib.sama_oracle_fd.argtypes = [C.c_int32, dp, dp, fp, C.c_double, C.c_int32, dp]
+    lib.sama_oracle_fd.restype = None
+    lib.sama_oracle_step.argtypes = [C.c_int32, ip, C.c_int64, fp, fp, fp, fp, fp, ap, C.c_double,
+                                     fp, ip, fp, C.c_int32, C.c_int32, dp, dp, dp, dp, dp, dp, dp]
+    lib.sama_oracle_step.restype = C.c_int
+    return lib
+
+
 def _load():
     global _lib
     if _lib is None:
-        lib = C.CDLL(build())
-        fp, dp, ip = C.POINTER(C.c_float), C.POINTER(C.c_double), C.POINTER(C.c_int32)
-        ap = C.POINTER(_Adam)
-        lib.sama_oracle_adapt.argtypes = [C.c_int64, fp, fp, fp, fp, ap, dp]
-        lib.sama_oracle_adapt.restype = None
-        lib.sama_oracle_sumsq.argtypes = [C.c_int64, dp]
-        lib.sama_oracle_sumsq.restype = C.c_double
-        lib.sama_oracle_perturb.argtypes = [C.c_int64, fp, dp, C.c_double, dp, dp, dp]
-        lib.sama_oracle_perturb.restype = C.c_int
-        lib.sama_oracle_losses.argtypes = [C.c_int32, ip, dp, fp, ip, C.c_int32, dp, dp]
-        lib.sama_oracle_losses.restype = None
-        lib.sama_oracle_fd.argtypes = [C.c_int32, dp, dp, fp, C.c_double, C.c_int32, dp]
-        lib.sama_oracle_fd.restype = None
-        lib.sama_oracle_step.argtypes = [C.c_int32, ip, C.c_int64, fp, fp, fp, fp, fp, ap, C.c_double,
-                                         fp, ip, fp, C.c_int32, C.c_int32, dp, dp, dp, dp, dp, dp, dp]
-        lib.sama_oracle_step.restype = C.c_int
-        _lib = lib
+        _lib = _bind(C.CDLL(build()))
     return _lib
 
 

@@ -1,0 +1,68 @@
+"""Checks that the pins have teeth: each plausible mistake, planted in a copy
+of the CPU checker's source, must make at least one pin fail."""
+import ctypes
+import os
+import subprocess
+
+import pytest
+
+import oracle
+import test_oracle_pins as pins
+
+MUTATIONS = {
+    "garbled_mg_coefficients": ("b1 * (1.0 - b2) * mk * g", "(1.0 - b1) * b2 * mk * g"),
+    "mg_term_sign": ("- b1 * (1.0 - b2) * mk * g", "+ b1 * (1.0 - b2) * mk * g"),
+    "eps_term_always_dropped": ("if (!h->drop_eps_term) num +=", "if (false) num +="),
+    "missing_sqrt_c2_in_denominator": ("num / (rc2 * r * D * D)", "num / (r * D * D)"),
+    "no_bias_correction_in_D": ("const double D = r / rc2 + eps;", "const double D = r + eps;"),
+    "missing_c1": ("J = (h->lr / c1) * num", "J = (h->lr) * num"),
+    "second_moment_uses_beta1": ("b2 * sk + (1.0 - b2) * g * g", "b1 * sk + (1.0 - b1) * g * g"),
+    "gbase_ignored": ("const double g = g_base ? (double)g_base[k] : mk;", "const double g = mk;"),
+    "minus_branch_sign": ("theta_minus[k] = t - d;", "theta_minus[k] = t + d;"),
+    "eps_from_squared_norm": ("bad ? 0.0 : alpha / norm;", "bad ? 0.0 : alpha / (norm * norm);"),
+    "transposed_weights": ("const double* w = W + (int64_t)j * din;\n                for (int32_t k = 0; k < din; ++k) acc += w[k] * h[k];",
+                           "for (int32_t k = 0; k < din; ++k) acc += W[(int64_t)k * dout + j] * h[k];"),
+    "relu_on_last_layer": ("(l + 1 < n_layers && acc < 0.0)", "(acc < 0.0)"),
+    "bias_dropped": ("double acc = b[j];", "double acc = 0.0 * b[j];"),
+    "wrong_label_logit": ("zmax - h[y[i]];", "zmax - h[0];"),
+    "no_max_shift_back": ("std::log(se) + zmax - h[y[i]]", "std::log(se) - h[y[i]]"),
+    "fd_sign": ("metagrad_out[i] = -sg", "metagrad_out[i] = sg"),
+    "fd_one_sided_scale": ("(2.0 * eps_fd * (double)B_norm)", "(eps_fd * (double)B_norm)"),
+    "sigmoid_instead_of_derivative": ("-sg * (1.0 - sg) *", "-sg *"),
+    "no_batch_mean": ("(2.0 * eps_fd * (double)B_norm)", "(2.0 * eps_fd)"),
+}
+
+PINS = [getattr(pins, n) for n in dir(pins) if n.startswith("test_")]
+
+
+def _run_all_pins():
+    failures = 0
+    for fn in PINS:
+        marks = [m for m in getattr(fn, "pytestmark", []) if m.name == "parametrize"]
+        argsets = [()]
+        if marks:
+            names = [a.strip() for a in marks[0].args[0].split(",")]
+            argsets = [v if len(names) > 1 else (v,) for v in marks[0].args[1]]
+        for args in argsets:
+            try:
+                fn(*args)
+            except AssertionError:
+                failures += 1
+    return failures
+
+
+def test_unmutated_checker_passes_every_pin():
+    assert _run_all_pins() == 0
+
+
+@pytest.mark.parametrize("name", sorted(MUTATIONS))
+def test_planted_mistake_is_caught(name, tmp_path, monkeypatch):
+    old, new = MUTATIONS[name]
+    src = open(os.path.join(os.path.dirname(oracle.__file__), "sama_oracle.cpp")).read()
+    assert src.count(old) == 1, "mutation site not found exactly once"
+    mutated = tmp_path / "mutant.cpp"
+    mutated.write_text(src.replace(old, new))
+    so = tmp_path / "mutant.so"
+    subprocess.check_call(["g++", "-O1", "-std=c++17", "-fPIC", "-shared", "-o", str(so), str(mutated)])
+    monkeypatch.setattr(oracle, "_lib", oracle._bind(ctypes.CDLL(str(so))))
+    assert _run_all_pins() > 0, "no pin noticed: " + name
