@@ -1,0 +1,188 @@
+/*
+ * sama.h -- C ABI of the B200 (sm_100a) SAMA meta-gradient library.
+ *
+ * SAMA ("Making Scalable Meta Learning Practical", arXiv 2310.05674) computes
+ * the meta gradient without second-order products:
+ *
+ *   p        = (du/dg_base) * g_meta             Eq. 4; Adam matrix: Appendix C
+ *   eps_fd   = alpha / ||p||_2                   Sec. 3.2
+ *   theta+-  = theta +- eps_fd * p               Sec. 3.2
+ *   dL_meta/dlambda ~= -[dL_base(theta+)/dlambda - dL_base(theta-)/dlambda] / (2 eps_fd)   Eq. 5
+ *
+ * Here lambda are per-sample weight logits of a data-reweighting objective
+ * (Sec. 4.1):  L_base = (1/B) sum_i sigmoid(lambda_i) * CE(f(x_i; theta), y_i),
+ * f an MLP, so Eq. 5 needs only per-sample losses at theta+ and theta-.
+ *
+ * Conventions
+ *   - Every array pointer is a DEVICE pointer owned by the caller unless the
+ *     argument is documented as "host".  The library never frees, reallocates
+ *     or keeps caller memory.  Structs (sama_adam_t, sama_mlp_t and the dims
+ *     array) are HOST memory, read during the call only.
+ *   - Arrays are fp32, contiguous.  Pointers need 4-byte alignment; 16-byte
+ *     alignment selects the vectorised kernels (same results).
+ *   - The flat parameter vector is W1, b1, W2, b2, ..., W_l stored
+ *     [d_l][d_{l-1}] row-major; the batch X is [B][d_0] row-major; labels are
+ *     int32 in [0, d_L).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
+ *     work is enqueued on it; no call synchronises unless it says so.
+ *   - Return value: SAMA_OK or a negative sama_status.  Argument errors are
+ *     detected on the host before anything is launched.  Conditions that only
+ *     the device can see (zero / non-finite ||p||, label out of range, an
+ *     internal wait that ran out) set bits in a device status word that
+ *     sama_device_status() reads; the kernels then write defined values
+ *     (theta+- = theta, metagrad = 0) instead of faulting.
+ *   - A context serialises nothing: calls that use the same context on
+ *     different streams at the same time race on its workspace.
+ */
+#ifndef SAMA_H
+#define SAMA_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum sama_status {
+    SAMA_OK = 0,
+    SAMA_ERR_NULL = -1,    /* a required pointer is NULL */
+    SAMA_ERR_ALIGN = -2,   /* a pointer is not aligned to its element type */
+    SAMA_ERR_SIZE = -3,    /* n < 0, n != parameter count of the MLP, B < 1, sizes beyond the context's limits */
+    SAMA_ERR_PARAM = -4,   /* step < 1 with bias correction, beta outside [0,1), non-finite or non-positive lr/eps/alpha */
+    SAMA_ERR_OVERLAP = -5, /* buffers overlap in a way that is not allowed */
+    SAMA_ERR_CUDA = -6,    /* a CUDA runtime call failed; see sama_last_cuda_error() */
+    SAMA_ERR_NOMEM = -7,   /* workspace allocation failed */
+    SAMA_ERR_UNSUPPORTED = -8
+} sama_status;
+
+/* Bits of the device status word. */
+enum {
+    SAMA_DEV_DEGENERATE_NORM = 1, /* ||p|| was 0 or not finite: eps_fd = 0, theta+- = theta, metagrad = 0 */
+    SAMA_DEV_BAD_LABEL = 2,       /* a label outside [0, d_L): that sample's metagrad is 0 */
+    SAMA_DEV_TIMEOUT = 4          /* a bounded wait inside a kernel expired; outputs of that call are invalid */
+};
+
+/* Base optimiser state that the adaptation differentiates (Appendix C).
+ * The update is u = (lr/c1) m' / (sqrt(s')/sqrt(c2) + eps) with
+ * m' = beta1 m + (1-beta1) g, s' = beta2 s + (1-beta2) g^2 and
+ * c1 = 1-beta1^step, c2 = 1-beta2^step.  (m, s) are the moments BEFORE this
+ * update; `step` >= 1 is the index of the update. */
+typedef struct sama_adam_t {
+    float lr, beta1, beta2, eps;
+    int64_t step;
+    int32_t bias_correction; /* 1: as above.  0: c1 = c2 = 1, the form printed in Appendix C */
+    int32_t drop_eps_term;   /* 0: exact derivative.  1: Appendix C's last line (eps-term of the numerator dropped) */
+    int32_t identity;        /* 1: du/dg = I (SGD base optimiser, Sec. 3.2; the SAMA-NA variant of Sec. 4.1) */
+} sama_adam_t;
+
+/* Base model: fully connected, ReLU between layers, last layer linear.
+ * dims (host) has n_layers + 1 entries d_0 .. d_L. */
+typedef struct sama_mlp_t {
+    int32_t n_layers;
+    const int32_t* dims;
+} sama_mlp_t;
+
+typedef struct sama_ctx sama_ctx;
+
+/* Creates a context on `device` with workspace for flat vectors up to max_n
+ * elements and, if `mlp` is given, for forward passes of that model (or any
+ * model whose widest layer and class count are not larger) on batches up to
+ * max_batch.  Allocates device memory; synchronises.  mlp may be NULL
+ * (adapt/perturb only). */
+int sama_create(sama_ctx** out, int device, int64_t max_n, int32_t max_batch, const sama_mlp_t* mlp);
+
+/* Frees the workspace.  The caller must have synchronised the streams used. */
+int sama_destroy(sama_ctx* ctx);
+
+/* Eq. 4 + Appendix C, fused with the squared norm of Sec. 3.2:
+ *   p_out[k] = J_k * g_meta[k],  J_k = du/dg at element k,  and  sum_k p_out[k]^2.
+ * m, s, g_meta: [n].  g_base: [n] or NULL (then g := m, the optimiser's own
+ * running estimate of the gradient).  p_out: [n]; may be the same pointer as
+ * g_meta (in place).  sumsq_out: one double on the device, or NULL; the sum
+ * is also left in the context (sama_ctx_sumsq).  The sum is accumulated in
+ * double in a fixed order: repeated calls give bit-identical results.
+ * n = 0 is allowed (sum = 0). */
+int sama_adapt(sama_ctx* ctx, int64_t n, const float* m, const float* s, const float* g_base,
+               const float* g_meta, const sama_adam_t* adam, float* p_out, double* sumsq_out, void* stream);
+
+/* Sec. 3.2: eps_fd = alpha / sqrt(sumsq);  theta_plus = theta + eps_fd p,
+ * theta_minus = theta - eps_fd p, written in one sweep.
+ * p_sumsq: device double holding sum p^2 (e.g. sama_adapt's), or NULL to have
+ * it computed here from p (one extra read of p).  theta_minus may be the same
+ * pointer as theta: that is the base-parameter nudge theta <- theta - eps_fd p
+ * the paper applies at each meta update (Sec. 3.2).  eps_fd_out: one float on
+ * the device, or NULL; eps_fd is also left in the context (sama_ctx_eps_fd).
+ * If the norm is 0 or not finite: eps_fd = 0, theta+- = theta,
+ * SAMA_DEV_DEGENERATE_NORM is set. */
+int sama_perturb(sama_ctx* ctx, int64_t n, const float* theta, const float* p, const double* p_sumsq,
+                 float alpha, float* theta_plus, float* theta_minus, float* eps_fd_out, void* stream);
+
+/* Eq. 5 for per-sample weight logits.  Runs the MLP on X at theta_plus and at
+ * theta_minus (both branches in the same launches), then
+ *   metagrad[i] = -sigmoid'(lambda_i) (loss+_i - loss-_i) / (2 eps_fd B),
+ *   loss_i = logsumexp(z_i) - z_i[y_i].
+ * theta_plus, theta_minus: [n_params(mlp)].  X: [B][d_0].  y: int32 [B].
+ * lambda: [B].  eps_fd: one float on the device (NULL: the context's, as left
+ * by the last sama_perturb).  metagrad_out: [B].  loss_plus_out,
+ * loss_minus_out: [B] or NULL.  All matrix products are carried out in
+ * arithmetic that is faithful to fp32 (the difference of the two branches is
+ * ~1e-3 of the losses, so reduced-precision products are not usable). */
+int sama_fd_metagrad(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const float* theta_minus,
+                     const float* X, const int32_t* y, const float* lambda, int32_t B, const float* eps_fd,
+                     float* metagrad_out, float* loss_plus_out, float* loss_minus_out, void* stream);
+
+/* The whole meta-gradient step of Fig. 2 with lambda = per-sample weights:
+ * sama_adapt -> sama_perturb -> sama_fd_metagrad on one stream, no host
+ * synchronisation in between.  n must equal the parameter count of mlp.
+ * Outputs: p_out [n] (may alias g_meta), theta_plus [n], theta_minus [n] (may
+ * alias theta), metagrad_out [B]; loss_*_out optional. */
+int sama_step(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* theta, const float* m,
+              const float* s, const float* g_base, const float* g_meta, const sama_adam_t* adam, float alpha,
+              const float* X, const int32_t* y, const float* lambda, int32_t B,
+              float* p_out, float* theta_plus, float* theta_minus, float* metagrad_out,
+              float* loss_plus_out, float* loss_minus_out, void* stream);
+
+/* sama_step (Fig. 2) for callers whose data lives in HOST memory: every
+ * pointer below is a host pointer (pinned memory makes the copies
+ * asynchronous).  Copies the inputs to staging buffers owned by the context
+ * (allocated on the first call, grown when needed), runs the step, copies
+ * metagrad (and eps_fd) back and synchronises `stream` before returning.
+ * theta_minus_out_host may be NULL; if given it receives theta - eps_fd p.
+ * Needs a context created with an mlp. */
+int sama_step_host(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* theta_host, const float* m_host,
+                   const float* s_host, const float* g_base_host, const float* g_meta_host,
+                   const sama_adam_t* adam, float alpha, const float* X_host, const int32_t* y_host,
+                   const float* lambda_host, int32_t B, float* metagrad_out_host, float* eps_fd_out_host,
+                   float* theta_minus_out_host, void* stream);
+
+/* Device addresses of the context's scalar slots of Sec. 3.2 (sum p^2 and
+ * eps_fd), valid until sama_destroy. */
+double* sama_ctx_sumsq(sama_ctx* ctx);
+float* sama_ctx_eps_fd(sama_ctx* ctx);
+
+/* Synchronises `stream`, returns the OR of the device status bits raised since
+ * the last call in *status_out and clears them. */
+int sama_device_status(sama_ctx* ctx, void* stream, int32_t* status_out);
+
+/* cudaError_t value of the last failed runtime call on this context (0 if none). */
+int sama_last_cuda_error(sama_ctx* ctx);
+
+/* Parameter count sum_l (d_{l-1} d_l + d_l), or -1 for an invalid description. */
+int64_t sama_mlp_param_count(const sama_mlp_t* mlp);
+
+/* Static text for a sama_status value. */
+const char* sama_status_string(int status);
+
+/* Selects how sama_fd_metagrad (Eq. 5) multiplies matrices: 0 = automatic,
+ * 1 = fp32 FMA on the CUDA cores, 2 = tensor cores with each fp32 operand
+ * split into two TF32 terms and three products per block (error comparable
+ * to fp32).  Returns SAMA_ERR_UNSUPPORTED for a mode this build lacks. */
+int sama_set_gemm_mode(sama_ctx* ctx, int mode);
+
+/* Number of kernels the library has launched through this context. */
+int64_t sama_launch_count(sama_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAMA_H */

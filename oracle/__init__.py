@@ -60,6 +60,8 @@ def _bind(lib):
     lib.sama_oracle_sumsq.restype = C.c_double
     lib.sama_oracle_perturb.argtypes = [C.c_int64, fp, dp, C.c_double, dp, dp, dp]
     lib.sama_oracle_perturb.restype = C.c_int
+    lib.sama_oracle_perturb_given_sumsq.argtypes = [C.c_int64, fp, dp, C.c_double, C.c_double, dp, dp, dp]
+    lib.sama_oracle_perturb_given_sumsq.restype = C.c_int
     lib.sama_oracle_losses.argtypes = [C.c_int32, ip, dp, fp, ip, C.c_int32, dp, dp]
     lib.sama_oracle_losses.restype = None
     lib.sama_oracle_fd.argtypes = [C.c_int32, dp, dp, fp, C.c_double, C.c_int32, dp]
@@ -118,6 +120,18 @@ def perturb(theta, p, alpha: float):
     eps = C.c_double(0.0)
     bad = _load().sama_oracle_perturb(n, _p(theta, C.c_float), _p(p, C.c_double), float(alpha),
                                       _p(tp, C.c_double), _p(tm, C.c_double), C.byref(eps))
+    return tp, tm, eps.value, bool(bad)
+
+
+def perturb_given_sumsq(theta, p, sumsq_all: float, alpha: float):
+    """S3 on a slice, with the sum of squares of the whole vector supplied."""
+    theta, p = _f32(theta), _f64(p)
+    n = theta.size
+    tp, tm = np.empty(n, dtype=np.float64), np.empty(n, dtype=np.float64)
+    eps = C.c_double(0.0)
+    bad = _load().sama_oracle_perturb_given_sumsq(n, _p(theta, C.c_float), _p(p, C.c_double), float(sumsq_all),
+                                                  float(alpha), _p(tp, C.c_double), _p(tm, C.c_double),
+                                                  C.byref(eps))
     return tp, tm, eps.value, bool(bad)
 
 

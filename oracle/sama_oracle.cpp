@@ -96,11 +96,13 @@ double sama_oracle_sumsq(int64_t n, const double* p) {
     return acc;
 }
 
-// S2 + S3 -- Sec. 3.2: eps_fd = alpha/||p||, theta+- = theta +- eps_fd p.
-// Returns 1 (and theta+- = theta, eps_fd = 0) when ||p|| is 0 or not finite.
-int sama_oracle_perturb(int64_t n, const float* theta, const double* p, double alpha,
-                        double* theta_plus, double* theta_minus, double* eps_fd_out) {
-    const double norm = std::sqrt(sama_oracle_sumsq(n, p));
+// S3 given S2's sum of squares -- Sec. 3.2: eps_fd = alpha/sqrt(sumsq),
+// theta+- = theta +- eps_fd p on the n elements given (which may be a slice of
+// the vector the sum was taken over).  Returns 1 (and theta+- = theta,
+// eps_fd = 0) when the norm is 0 or not finite.
+int sama_oracle_perturb_given_sumsq(int64_t n, const float* theta, const double* p, double sumsq, double alpha,
+                                    double* theta_plus, double* theta_minus, double* eps_fd_out) {
+    const double norm = std::sqrt(sumsq);
     const bool bad = !(norm > 0.0) || !std::isfinite(norm);
     const double eps_fd = bad ? 0.0 : alpha / norm;
     for (int64_t k = 0; k < n; ++k) {
@@ -111,6 +113,13 @@ int sama_oracle_perturb(int64_t n, const float* theta, const double* p, double a
     }
     *eps_fd_out = eps_fd;
     return bad ? 1 : 0;
+}
+
+// S2 + S3 -- Sec. 3.2 on a whole vector.
+int sama_oracle_perturb(int64_t n, const float* theta, const double* p, double alpha,
+                        double* theta_plus, double* theta_minus, double* eps_fd_out) {
+    return sama_oracle_perturb_given_sumsq(n, theta, p, sama_oracle_sumsq(n, p), alpha, theta_plus, theta_minus,
+                                           eps_fd_out);
 }
 
 // S4 -- per-sample cross-entropy of the base MLP at parameters theta.

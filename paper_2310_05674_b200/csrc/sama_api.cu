@@ -1,0 +1,456 @@
+// Host side of the C ABI: argument validation, workspace, launch sequencing.
+// Every step of the SAMA update runs in the kernels; nothing here computes on
+// the CPU beyond the scalar constants of the Adam adaptation matrix.
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "sama_internal.h"
+
+using namespace sama;
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+inline int cuda_fail(sama_ctx* ctx, cudaError_t e) {
+    if (ctx) ctx->last_cuda_error = (int)e;
+    return SAMA_ERR_CUDA;
+}
+#define SAMA_CUDA(ctx, expr)                                   \
+    do {                                                       \
+        cudaError_t e__ = (expr);                              \
+        if (e__ != cudaSuccess) return cuda_fail((ctx), e__);  \
+    } while (0)
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// true if [a, a+na) and [b, b+nb) share a byte
+inline bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+    if (!a || !b || na == 0 || nb == 0) return false;
+    const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+    return x < y + nb && y < x + na;
+}
+
+int check_mlp(const sama_mlp_t* mlp) {
+    if (!mlp || !mlp->dims) return SAMA_ERR_NULL;
+    if (mlp->n_layers < 1 || mlp->n_layers > kMaxLayers) return SAMA_ERR_SIZE;
+    for (int l = 0; l <= mlp->n_layers; ++l)
+        if (mlp->dims[l] < 1) return SAMA_ERR_SIZE;
+    return SAMA_OK;
+}
+
+int check_adam(const sama_adam_t* a, AdaptConsts* out) {
+    if (!a) return SAMA_ERR_NULL;
+    AdaptConsts c;
+    std::memset(&c, 0, sizeof(c));
+    c.identity = a->identity ? 1 : 0;
+    c.drop_eps_term = a->drop_eps_term ? 1 : 0;
+    if (!c.identity) {
+        if (!(a->beta1 >= 0.f && a->beta1 < 1.f) || !(a->beta2 >= 0.f && a->beta2 < 1.f)) return SAMA_ERR_PARAM;
+        if (!std::isfinite(a->lr) || !(a->lr > 0.f)) return SAMA_ERR_PARAM;
+        if (!std::isfinite(a->eps) || !(a->eps >= 0.f)) return SAMA_ERR_PARAM;
+        double c1 = 1.0, c2 = 1.0;
+        if (a->bias_correction) {
+            if (a->step < 1) return SAMA_ERR_PARAM;
+            c1 = 1.0 - std::pow((double)a->beta1, (double)a->step);
+            c2 = 1.0 - std::pow((double)a->beta2, (double)a->step);
+            if (!(c1 > 0.0) || !(c2 > 0.0)) return SAMA_ERR_PARAM;
+        }
+        c.a = (float)((double)a->lr / c1);
+        c.b1 = a->beta1;
+        c.b2 = a->beta2;
+        c.omb1 = (float)(1.0 - (double)a->beta1);
+        c.omb2 = (float)(1.0 - (double)a->beta2);
+        c.inv_rc2 = (float)(1.0 / std::sqrt(c2));
+        c.eps = a->eps;
+    }
+    *out = c;
+    return SAMA_OK;
+}
+
+int validate_adapt(sama_ctx* ctx, int64_t n, const float* m, const float* s, const float* g_base,
+                   const float* g_meta, const sama_adam_t* adam, float* p_out, double* sumsq_out,
+                   AdaptConsts* c) {
+    if (!ctx || !adam || !g_meta || !p_out) return SAMA_ERR_NULL;
+    const int rc = check_adam(adam, c);
+    if (rc != SAMA_OK) return rc;
+    if (!c->identity && (!m || !s)) return SAMA_ERR_NULL;
+    if (n < 0 || n > ctx->max_n) return SAMA_ERR_SIZE;
+    if (!aligned(m, 4) || !aligned(s, 4) || !aligned(g_base, 4) || !aligned(g_meta, 4) || !aligned(p_out, 4) ||
+        !aligned(sumsq_out, 8))
+        return SAMA_ERR_ALIGN;
+    const size_t bytes = (size_t)n * 4;
+    if (overlaps(p_out, bytes, m, bytes) || overlaps(p_out, bytes, s, bytes) ||
+        overlaps(p_out, bytes, g_base, bytes) || overlaps(p_out, bytes, sumsq_out, 8))
+        return SAMA_ERR_OVERLAP;
+    if (p_out != g_meta && overlaps(p_out, bytes, g_meta, bytes)) return SAMA_ERR_OVERLAP;
+    return SAMA_OK;
+}
+
+int validate_perturb(sama_ctx* ctx, int64_t n, const float* theta, const float* p, const double* p_sumsq,
+                     float alpha, float* theta_plus, float* theta_minus, float* eps_fd_out) {
+    if (!ctx || !theta || !p || !theta_plus || !theta_minus) return SAMA_ERR_NULL;
+    if (n < 0 || n > ctx->max_n) return SAMA_ERR_SIZE;
+    if (!std::isfinite(alpha) || !(alpha > 0.f)) return SAMA_ERR_PARAM;
+    if (!aligned(theta, 4) || !aligned(p, 4) || !aligned(theta_plus, 4) || !aligned(theta_minus, 4) ||
+        !aligned(p_sumsq, 8) || !aligned(eps_fd_out, 4))
+        return SAMA_ERR_ALIGN;
+    const size_t bytes = (size_t)n * 4;
+    if (overlaps(theta_plus, bytes, theta_minus, bytes) || overlaps(theta_plus, bytes, theta, bytes) ||
+        overlaps(theta_plus, bytes, p, bytes) || overlaps(theta_minus, bytes, p, bytes) ||
+        overlaps(theta_plus, bytes, eps_fd_out, 4) || overlaps(theta_minus, bytes, eps_fd_out, 4) ||
+        overlaps(theta_plus, bytes, p_sumsq, 8) || overlaps(theta_minus, bytes, p_sumsq, 8))
+        return SAMA_ERR_OVERLAP;
+    if (theta_minus != theta && overlaps(theta_minus, bytes, theta, bytes)) return SAMA_ERR_OVERLAP;
+    return SAMA_OK;
+}
+
+int validate_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const float* theta_minus,
+                const float* X, const int32_t* y, const float* lambda, int32_t B, const float* eps_fd,
+                float* metagrad_out, float* loss_plus_out, float* loss_minus_out) {
+    if (!ctx || !theta_plus || !theta_minus || !X || !y || !lambda || !metagrad_out) return SAMA_ERR_NULL;
+    const int rc = check_mlp(mlp);
+    if (rc != SAMA_OK) return rc;
+    if (B < 1 || B > ctx->max_batch || ctx->max_classes == 0) return SAMA_ERR_SIZE;
+    const int L = mlp->n_layers;
+    for (int l = 1; l < L; ++l)
+        if (mlp->dims[l] > ctx->max_width) return SAMA_ERR_SIZE;
+    if (mlp->dims[L] > ctx->max_classes) return SAMA_ERR_SIZE;
+    if (!aligned(theta_plus, 4) || !aligned(theta_minus, 4) || !aligned(X, 4) || !aligned(y, 4) ||
+        !aligned(lambda, 4) || !aligned(eps_fd, 4) || !aligned(metagrad_out, 4) || !aligned(loss_plus_out, 4) ||
+        !aligned(loss_minus_out, 4))
+        return SAMA_ERR_ALIGN;
+    const size_t nb = (size_t)sama_mlp_param_count(mlp) * 4, bb = (size_t)B * 4;
+    float* outs[3] = {metagrad_out, loss_plus_out, loss_minus_out};
+    for (int i = 0; i < 3; ++i) {
+        if (!outs[i]) continue;
+        if (overlaps(outs[i], bb, theta_plus, nb) || overlaps(outs[i], bb, theta_minus, nb) ||
+            overlaps(outs[i], bb, X, (size_t)B * mlp->dims[0] * 4) || overlaps(outs[i], bb, y, bb) ||
+            overlaps(outs[i], bb, lambda, bb) || overlaps(outs[i], bb, eps_fd, 4))
+            return SAMA_ERR_OVERLAP;
+        for (int j = i + 1; j < 3; ++j)
+            if (overlaps(outs[i], bb, outs[j], bb)) return SAMA_ERR_OVERLAP;
+    }
+    return SAMA_OK;
+}
+
+// The dual-branch forward and the finite difference, arguments already validated.
+int run_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const float* theta_minus,
+           const float* X, const int32_t* y, const float* lambda, int32_t B, const float* eps_fd,
+           float* metagrad_out, float* loss_plus_out, float* loss_minus_out, cudaStream_t st) {
+    const int L = mlp->n_layers;
+    const float* in[2] = {X, X};
+    int ld_in = mlp->dims[0];
+    int64_t off = 0;
+    for (int l = 0; l < L; ++l) {
+        const int din = mlp->dims[l], dout = mlp->dims[l + 1];
+        const bool last = (l + 1 == L);
+        float* out0 = last ? ctx->logits : ctx->act[l & 1];
+        GemmArgs g;
+        g.A[0] = in[0];
+        g.A[1] = in[1];
+        g.W[0] = theta_plus + off;
+        g.W[1] = theta_minus + off;
+        g.bias[0] = theta_plus + off + (int64_t)din * dout;
+        g.bias[1] = theta_minus + off + (int64_t)din * dout;
+        g.C[0] = out0;
+        g.C[1] = out0 + (int64_t)B * dout;
+        g.M = B;
+        g.N = dout;
+        g.K = din;
+        g.lda = ld_in;
+        g.ldw = din;
+        g.ldc = dout;
+        g.relu = last ? 0 : 1;
+        SAMA_CUDA(ctx, launch_gemm(ctx, g, st));
+        in[0] = g.C[0];
+        in[1] = g.C[1];
+        ld_in = dout;
+        off += (int64_t)din * dout + dout;
+    }
+    const int C = mlp->dims[L];
+    SAMA_CUDA(ctx, launch_ce_fd(ctx, in[0], in[1], C, y, lambda, B, C, eps_fd ? eps_fd : &ctx->scalars->eps_fd,
+                                metagrad_out, loss_plus_out, loss_minus_out, st));
+    return SAMA_OK;
+}
+
+}  // namespace
+
+namespace sama {
+cudaError_t launch_gemm(sama_ctx* ctx, const GemmArgs& g, cudaStream_t st) {
+    return launch_gemm_ffma(ctx, g, st);
+}
+}  // namespace sama
+
+extern "C" {
+
+int64_t sama_mlp_param_count(const sama_mlp_t* mlp) {
+    if (check_mlp(mlp) != SAMA_OK) return -1;
+    int64_t n = 0;
+    for (int l = 0; l < mlp->n_layers; ++l) n += (int64_t)mlp->dims[l] * mlp->dims[l + 1] + mlp->dims[l + 1];
+    return n;
+}
+
+int sama_create(sama_ctx** out, int device, int64_t max_n, int32_t max_batch, const sama_mlp_t* mlp) {
+    if (!out) return SAMA_ERR_NULL;
+    *out = nullptr;
+    if (max_n < 0 || max_batch < 0) return SAMA_ERR_SIZE;
+    if (mlp) {
+        const int rc = check_mlp(mlp);
+        if (rc != SAMA_OK) return rc;
+        if (max_batch < 1) return SAMA_ERR_SIZE;
+    }
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+        cudaGetLastError();
+        return SAMA_ERR_CUDA;
+    }
+    DeviceGuard guard(device);
+    if (!guard.ok) return SAMA_ERR_CUDA;
+    sama_ctx* ctx = new (std::nothrow) sama_ctx();
+    if (!ctx) return SAMA_ERR_NOMEM;
+    std::memset(ctx, 0, sizeof(*ctx));
+    ctx->device = device;
+    ctx->max_n = max_n;
+    ctx->max_batch = max_batch;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return SAMA_ERR_CUDA; }
+    ctx->sm_count = prop.multiProcessorCount;
+    bool ok = cudaMalloc(&ctx->scalars, sizeof(DeviceScalars)) == cudaSuccess &&
+              cudaMemset(ctx->scalars, 0, sizeof(DeviceScalars)) == cudaSuccess &&
+              cudaMalloc(&ctx->partials, sizeof(double) * kMaxPartials) == cudaSuccess;
+    if (ok && mlp) {
+        const int L = mlp->n_layers;
+        int width = 0;
+        for (int l = 1; l < L; ++l) width = mlp->dims[l] > width ? mlp->dims[l] : width;
+        ctx->max_width = width;
+        ctx->max_classes = mlp->dims[L];
+        if (width > 0) {
+            const size_t bytes = sizeof(float) * 2 * (size_t)max_batch * width;
+            ok = cudaMalloc(&ctx->act[0], bytes) == cudaSuccess && cudaMalloc(&ctx->act[1], bytes) == cudaSuccess;
+        }
+        ok = ok && cudaMalloc(&ctx->logits, sizeof(float) * 2 * (size_t)max_batch * ctx->max_classes) == cudaSuccess;
+    }
+    if (!ok || cudaDeviceSynchronize() != cudaSuccess) {
+        cudaGetLastError();
+        sama_destroy(ctx);
+        return SAMA_ERR_NOMEM;
+    }
+    *out = ctx;
+    return SAMA_OK;
+}
+
+int sama_destroy(sama_ctx* ctx) {
+    if (!ctx) return SAMA_OK;
+    DeviceGuard guard(ctx->device);
+    cudaFree(ctx->scalars);
+    cudaFree(ctx->partials);
+    cudaFree(ctx->act[0]);
+    cudaFree(ctx->act[1]);
+    cudaFree(ctx->logits);
+    cudaFree(ctx->stage);
+    delete ctx;
+    return SAMA_OK;
+}
+
+int sama_adapt(sama_ctx* ctx, int64_t n, const float* m, const float* s, const float* g_base,
+               const float* g_meta, const sama_adam_t* adam, float* p_out, double* sumsq_out, void* stream) {
+    AdaptConsts c;
+    const int rc = validate_adapt(ctx, n, m, s, g_base, g_meta, adam, p_out, sumsq_out, &c);
+    if (rc != SAMA_OK) return rc;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SAMA_ERR_CUDA;
+    SAMA_CUDA(ctx, launch_adapt_sumsq(ctx, n, m, s, c.identity ? nullptr : g_base, g_meta, c, p_out, sumsq_out,
+                                      (cudaStream_t)stream));
+    return SAMA_OK;
+}
+
+int sama_perturb(sama_ctx* ctx, int64_t n, const float* theta, const float* p, const double* p_sumsq,
+                 float alpha, float* theta_plus, float* theta_minus, float* eps_fd_out, void* stream) {
+    const int rc = validate_perturb(ctx, n, theta, p, p_sumsq, alpha, theta_plus, theta_minus, eps_fd_out);
+    if (rc != SAMA_OK) return rc;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SAMA_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!p_sumsq) {
+        SAMA_CUDA(ctx, launch_sumsq(ctx, n, p, st));
+        p_sumsq = &ctx->scalars->sumsq;
+    }
+    SAMA_CUDA(ctx, launch_perturb(ctx, n, theta, p, p_sumsq, alpha, theta_plus, theta_minus, eps_fd_out, st));
+    return SAMA_OK;
+}
+
+int sama_fd_metagrad(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const float* theta_minus,
+                     const float* X, const int32_t* y, const float* lambda, int32_t B, const float* eps_fd,
+                     float* metagrad_out, float* loss_plus_out, float* loss_minus_out, void* stream) {
+    const int rc = validate_fd(ctx, mlp, theta_plus, theta_minus, X, y, lambda, B, eps_fd, metagrad_out,
+                               loss_plus_out, loss_minus_out);
+    if (rc != SAMA_OK) return rc;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SAMA_ERR_CUDA;
+    return run_fd(ctx, mlp, theta_plus, theta_minus, X, y, lambda, B, eps_fd, metagrad_out, loss_plus_out,
+                  loss_minus_out, (cudaStream_t)stream);
+}
+
+int sama_step(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* theta, const float* m,
+              const float* s, const float* g_base, const float* g_meta, const sama_adam_t* adam, float alpha,
+              const float* X, const int32_t* y, const float* lambda, int32_t B,
+              float* p_out, float* theta_plus, float* theta_minus, float* metagrad_out,
+              float* loss_plus_out, float* loss_minus_out, void* stream) {
+    if (!ctx) return SAMA_ERR_NULL;
+    int rc = check_mlp(mlp);
+    if (rc != SAMA_OK) return rc;
+    if (n != sama_mlp_param_count(mlp)) return SAMA_ERR_SIZE;
+    AdaptConsts c;
+    rc = validate_adapt(ctx, n, m, s, g_base, g_meta, adam, p_out, nullptr, &c);
+    if (rc != SAMA_OK) return rc;
+    rc = validate_perturb(ctx, n, theta, p_out, nullptr, alpha, theta_plus, theta_minus, nullptr);
+    if (rc != SAMA_OK) return rc;
+    rc = validate_fd(ctx, mlp, theta_plus, theta_minus, X, y, lambda, B, nullptr, metagrad_out, loss_plus_out,
+                     loss_minus_out);
+    if (rc != SAMA_OK) return rc;
+    // outputs of the early stages must not be inputs of the later ones
+    const size_t nb = (size_t)n * 4, bb = (size_t)B * 4;
+    const void* ins[6] = {m, s, g_base, X, lambda, y};
+    const size_t inb[6] = {nb, nb, nb, (size_t)B * mlp->dims[0] * 4, bb, bb};
+    for (int i = 0; i < 6; ++i)
+        if (overlaps(theta_plus, nb, ins[i], inb[i]) || overlaps(theta_minus, nb, ins[i], inb[i]) ||
+            (i >= 3 && overlaps(p_out, nb, ins[i], inb[i])))
+            return SAMA_ERR_OVERLAP;
+    if (overlaps(theta_plus, nb, g_meta, nb) || overlaps(theta_minus, nb, g_meta, nb) ||
+        overlaps(p_out, nb, theta, nb))
+        return SAMA_ERR_OVERLAP;
+    float* outs[3] = {metagrad_out, loss_plus_out, loss_minus_out};
+    for (int i = 0; i < 3; ++i)
+        if (overlaps(outs[i], bb, p_out, nb) || overlaps(outs[i], bb, theta, nb) ||
+            overlaps(outs[i], bb, g_meta, nb) || overlaps(outs[i], bb, m, nb) || overlaps(outs[i], bb, s, nb) ||
+            overlaps(outs[i], bb, g_base, nb))
+            return SAMA_ERR_OVERLAP;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SAMA_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    SAMA_CUDA(ctx, launch_adapt_sumsq(ctx, n, m, s, c.identity ? nullptr : g_base, g_meta, c, p_out, nullptr, st));
+    SAMA_CUDA(ctx, launch_perturb(ctx, n, theta, p_out, &ctx->scalars->sumsq, alpha, theta_plus, theta_minus,
+                                  nullptr, st));
+    return run_fd(ctx, mlp, theta_plus, theta_minus, X, y, lambda, B, nullptr, metagrad_out, loss_plus_out,
+                  loss_minus_out, st);
+}
+
+int sama_step_host(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* theta_host, const float* m_host,
+                   const float* s_host, const float* g_base_host, const float* g_meta_host,
+                   const sama_adam_t* adam, float alpha, const float* X_host, const int32_t* y_host,
+                   const float* lambda_host, int32_t B, float* metagrad_out_host, float* eps_fd_out_host,
+                   float* theta_minus_out_host, void* stream) {
+    if (!ctx || !theta_host || !g_meta_host || !X_host || !y_host || !lambda_host || !metagrad_out_host || !adam)
+        return SAMA_ERR_NULL;
+    int rc = check_mlp(mlp);
+    if (rc != SAMA_OK) return rc;
+    if (n != sama_mlp_param_count(mlp) || n > ctx->max_n || B < 1 || B > ctx->max_batch) return SAMA_ERR_SIZE;
+    if (!adam->identity && (!m_host || !s_host)) return SAMA_ERR_NULL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SAMA_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    // staging layout (floats): theta m s g_base g_meta p theta+ theta- | X | lambda | metagrad | y
+    const size_t nn = ((size_t)n + 63) & ~(size_t)63;
+    const size_t xs = (((size_t)B * mlp->dims[0]) + 63) & ~(size_t)63;
+    const size_t bs = ((size_t)B + 63) & ~(size_t)63;
+    const size_t need = (8 * nn + xs + 3 * bs) * sizeof(float);
+    if (ctx->stage_bytes < need) {
+        SAMA_CUDA(ctx, cudaStreamSynchronize(st));
+        cudaFree(ctx->stage);
+        ctx->stage = nullptr;
+        ctx->stage_bytes = 0;
+        if (cudaMalloc(&ctx->stage, need) != cudaSuccess) { cudaGetLastError(); return SAMA_ERR_NOMEM; }
+        ctx->stage_bytes = need;
+    }
+    float* d_theta = ctx->stage;
+    float* d_m = d_theta + nn;
+    float* d_s = d_m + nn;
+    float* d_g = d_s + nn;
+    float* d_gm = d_g + nn;
+    float* d_p = d_gm + nn;
+    float* d_tp = d_p + nn;
+    float* d_tm = d_tp + nn;
+    float* d_X = d_tm + nn;
+    float* d_lam = d_X + xs;
+    float* d_mg = d_lam + bs;
+    int32_t* d_y = reinterpret_cast<int32_t*>(d_mg + bs);
+    const size_t nb = (size_t)n * 4;
+    SAMA_CUDA(ctx, cudaMemcpyAsync(d_theta, theta_host, nb, cudaMemcpyHostToDevice, st));
+    if (m_host) SAMA_CUDA(ctx, cudaMemcpyAsync(d_m, m_host, nb, cudaMemcpyHostToDevice, st));
+    if (s_host) SAMA_CUDA(ctx, cudaMemcpyAsync(d_s, s_host, nb, cudaMemcpyHostToDevice, st));
+    if (g_base_host) SAMA_CUDA(ctx, cudaMemcpyAsync(d_g, g_base_host, nb, cudaMemcpyHostToDevice, st));
+    SAMA_CUDA(ctx, cudaMemcpyAsync(d_gm, g_meta_host, nb, cudaMemcpyHostToDevice, st));
+    SAMA_CUDA(ctx, cudaMemcpyAsync(d_X, X_host, (size_t)B * mlp->dims[0] * 4, cudaMemcpyHostToDevice, st));
+    SAMA_CUDA(ctx, cudaMemcpyAsync(d_y, y_host, (size_t)B * 4, cudaMemcpyHostToDevice, st));
+    SAMA_CUDA(ctx, cudaMemcpyAsync(d_lam, lambda_host, (size_t)B * 4, cudaMemcpyHostToDevice, st));
+    rc = sama_step(ctx, mlp, n, d_theta, m_host ? d_m : nullptr, s_host ? d_s : nullptr,
+                   g_base_host ? d_g : nullptr, d_gm, adam, alpha, d_X, d_y, d_lam, B, d_p, d_tp, d_tm, d_mg,
+                   nullptr, nullptr, stream);
+    if (rc != SAMA_OK) return rc;
+    SAMA_CUDA(ctx, cudaMemcpyAsync(metagrad_out_host, d_mg, (size_t)B * 4, cudaMemcpyDeviceToHost, st));
+    if (eps_fd_out_host)
+        SAMA_CUDA(ctx, cudaMemcpyAsync(eps_fd_out_host, &ctx->scalars->eps_fd, 4, cudaMemcpyDeviceToHost, st));
+    if (theta_minus_out_host)
+        SAMA_CUDA(ctx, cudaMemcpyAsync(theta_minus_out_host, d_tm, nb, cudaMemcpyDeviceToHost, st));
+    SAMA_CUDA(ctx, cudaStreamSynchronize(st));
+    return SAMA_OK;
+}
+
+double* sama_ctx_sumsq(sama_ctx* ctx) { return ctx ? &ctx->scalars->sumsq : nullptr; }
+float* sama_ctx_eps_fd(sama_ctx* ctx) { return ctx ? &ctx->scalars->eps_fd : nullptr; }
+
+int sama_device_status(sama_ctx* ctx, void* stream, int32_t* status_out) {
+    if (!ctx || !status_out) return SAMA_ERR_NULL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SAMA_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    int32_t v = 0;
+    SAMA_CUDA(ctx, cudaMemcpyAsync(&v, &ctx->scalars->status, 4, cudaMemcpyDeviceToHost, st));
+    SAMA_CUDA(ctx, cudaMemsetAsync(&ctx->scalars->status, 0, 4, st));
+    SAMA_CUDA(ctx, cudaStreamSynchronize(st));
+    *status_out = v;
+    return SAMA_OK;
+}
+
+int sama_last_cuda_error(sama_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+int sama_set_gemm_mode(sama_ctx* ctx, int mode) {
+    if (!ctx) return SAMA_ERR_NULL;
+    if (mode < 0 || mode > 2) return SAMA_ERR_PARAM;
+    if (mode == 2) return SAMA_ERR_UNSUPPORTED;
+    ctx->gemm_mode = mode;
+    return SAMA_OK;
+}
+
+int64_t sama_launch_count(sama_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* sama_status_string(int status) {
+    switch (status) {
+        case SAMA_OK: return "ok";
+        case SAMA_ERR_NULL: return "a required pointer is NULL";
+        case SAMA_ERR_ALIGN: return "a pointer is not aligned to its element type";
+        case SAMA_ERR_SIZE: return "a size is negative, inconsistent or beyond the context's limits";
+        case SAMA_ERR_PARAM: return "a scalar parameter is out of range or not finite";
+        case SAMA_ERR_OVERLAP: return "buffers overlap in a way that is not allowed";
+        case SAMA_ERR_CUDA: return "a CUDA runtime call failed";
+        case SAMA_ERR_NOMEM: return "workspace allocation failed";
+        case SAMA_ERR_UNSUPPORTED: return "not supported by this build";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

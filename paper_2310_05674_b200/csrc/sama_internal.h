@@ -1,0 +1,84 @@
+// Internal declarations shared by the translation units of libsama.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sama.h"
+
+namespace sama {
+
+constexpr int kMaxLayers = 16;
+constexpr int kMaxPartials = 4096;  // upper bound on the grid of the reduction kernels
+
+// Device scalars owned by a context.
+struct DeviceScalars {
+    double sumsq;          // sum p^2 of the last adapt
+    float eps_fd;          // alpha / ||p|| of the last perturb
+    int32_t status;        // OR of SAMA_DEV_* bits
+    unsigned int counter;  // arrival counter of the last-block-done reduction (returns to 0)
+    unsigned int pad;
+};
+
+// Host-precomputed constants of the Adam adaptation matrix (Appendix C).
+struct AdaptConsts {
+    float a;        // lr / c1
+    float b1, b2;   // beta1, beta2
+    float omb1;     // 1 - beta1
+    float omb2;     // 1 - beta2
+    float inv_rc2;  // 1 / sqrt(c2)
+    float eps;      // Adam's epsilon
+    int drop_eps_term;
+    int identity;
+};
+
+}  // namespace sama
+
+struct sama_ctx {
+    int device;
+    int sm_count;
+    int64_t max_n;
+    int32_t max_batch;
+    int32_t max_width;    // widest hidden layer the forward workspace covers, 0 if none
+    int32_t max_classes;  // largest d_L covered, 0 if the context has no forward workspace
+    int gemm_mode;        // 0 auto, 1 ffma, 2 3xTF32
+    int last_cuda_error;
+    int64_t launches;
+    sama::DeviceScalars* scalars;  // device
+    double* partials;              // device [kMaxPartials]
+    float* act[2];                 // device: ping-pong activations, each [2][max_batch][max_width]
+    float* logits;                 // device [2][max_batch][max_classes]
+    float* stage;                  // device: staging of the host entry point (allocated on first use)
+    size_t stage_bytes;
+};
+
+namespace sama {
+
+// adapt_perturb.cu
+cudaError_t launch_adapt_sumsq(sama_ctx* ctx, int64_t n, const float* m, const float* s, const float* g_base,
+                               const float* g_meta, const AdaptConsts& c, float* p_out, double* sumsq_out,
+                               cudaStream_t st);
+cudaError_t launch_sumsq(sama_ctx* ctx, int64_t n, const float* p, cudaStream_t st);
+cudaError_t launch_perturb(sama_ctx* ctx, int64_t n, const float* theta, const float* p, const double* sumsq,
+                           float alpha, float* theta_plus, float* theta_minus, float* eps_fd_out, cudaStream_t st);
+
+// One layer of both branches: C[b] = act(A[b] * W[b]^T + bias[b]) for b in {0, 1}
+struct GemmArgs {
+    const float* A[2];     // [M][lda]
+    const float* W[2];     // [N][ldw]
+    const float* bias[2];  // [N]
+    float* C[2];           // [M][ldc]
+    int M, N, K;
+    int lda, ldw, ldc;
+    int relu;
+};
+// gemm_ffma.cu
+cudaError_t launch_gemm_ffma(sama_ctx* ctx, const GemmArgs& g, cudaStream_t st);
+// sama_api.cu : picks the matrix-product path of one layer
+cudaError_t launch_gemm(sama_ctx* ctx, const GemmArgs& g, cudaStream_t st);
+
+// ce_fd.cu
+cudaError_t launch_ce_fd(sama_ctx* ctx, const float* z_plus, const float* z_minus, int ldz, const int32_t* y,
+                         const float* lambda, int B, int C, const float* eps_fd, float* metagrad,
+                         float* loss_plus, float* loss_minus, cudaStream_t st);
+
+}  // namespace sama
