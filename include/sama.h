@@ -182,6 +182,34 @@ int sama_set_gemm_mode(sama_ctx* ctx, int mode);
 /* Number of kernels the library has launched through this context. */
 int64_t sama_launch_count(sama_ctx* ctx);
 
+/* Per-kernel timing.  While enabled, the library records a pair of CUDA events
+ * around every kernel it launches through this context, on the stream the
+ * kernel is launched on.  The kinds name the stages of the step: adaptation +
+ * norm (Eq. 4, Sec. 3.2), norm alone, perturbation (Sec. 3.2), one layer of
+ * the dual-branch forward pass, cross-entropy + central difference (Eq. 5). */
+enum {
+    SAMA_K_ADAPT = 0,
+    SAMA_K_SUMSQ = 1,
+    SAMA_K_PERTURB = 2,
+    SAMA_K_GEMM_FFMA = 3,
+    SAMA_K_CE_FD = 4,
+    SAMA_K_SPLIT = 5,
+    SAMA_K_GEMM_TF32X3 = 6
+};
+typedef struct sama_kernel_time_t {
+    int32_t kind;  /* SAMA_K_* */
+    int32_t layer; /* layer index for the forward kernels, else -1 */
+    float ms;      /* device time between the two events */
+} sama_kernel_time_t;
+
+/* on != 0: start recording (discarding earlier records); on == 0: stop and discard. */
+int sama_profile_enable(sama_ctx* ctx, int32_t on);
+
+/* Waits for the recorded events, writes up to `capacity` records (launch
+ * order) to the host array `out`, stores the number of records taken in
+ * *count_out and clears them.  Recording stays enabled. */
+int sama_profile_collect(sama_ctx* ctx, sama_kernel_time_t* out, int32_t capacity, int32_t* count_out);
+
 #ifdef __cplusplus
 }
 #endif

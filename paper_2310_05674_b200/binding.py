@@ -42,6 +42,14 @@ class sama_adam_t(C.Structure):
                 ("identity", C.c_int32)]
 
 
+class sama_kernel_time_t(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("layer", C.c_int32), ("ms", C.c_float)]
+
+
+KERNEL_KINDS = {0: "adapt_sumsq", 1: "sumsq", 2: "perturb", 3: "gemm_ffma", 4: "ce_fd", 5: "split_tf32",
+                6: "gemm_tf32x3"}
+
+
 class sama_mlp_t(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("dims", C.POINTER(C.c_int32))]
 
@@ -98,6 +106,8 @@ lib.sama_status_string.restype = C.c_char_p
 lib.sama_set_gemm_mode.argtypes = [_vp, C.c_int]
 lib.sama_launch_count.argtypes = [_vp]
 lib.sama_launch_count.restype = C.c_int64
+lib.sama_profile_enable.argtypes = [_vp, C.c_int32]
+lib.sama_profile_collect.argtypes = [_vp, C.POINTER(sama_kernel_time_t), C.c_int32, C.POINTER(C.c_int32)]
 
 
 def _ptr(x) -> Optional[int]:
@@ -206,3 +216,15 @@ def sama_set_gemm_mode(ctx, mode: int) -> int:
 
 def sama_launch_count(ctx) -> int:
     return int(lib.sama_launch_count(ctx))
+
+
+def sama_profile_enable(ctx, on: bool) -> int:
+    return _check(lib.sama_profile_enable(ctx, int(bool(on))), "sama_profile_enable")
+
+
+def sama_profile_collect(ctx, capacity: int = 65536):
+    """Returns [(kind, layer, ms), ...] in launch order."""
+    buf = (sama_kernel_time_t * capacity)()
+    cnt = C.c_int32(0)
+    _check(lib.sama_profile_collect(ctx, buf, capacity, C.byref(cnt)), "sama_profile_collect")
+    return [(buf[i].kind, buf[i].layer, buf[i].ms) for i in range(cnt.value)]

@@ -286,6 +286,7 @@ cudaError_t launch_adapt_sumsq(sama_ctx* ctx, int64_t n, const float* m, const f
                                cudaStream_t st) {
     const bool vec = aligned16(m) && aligned16(s) && aligned16(g_meta) && aligned16(p_out) &&
                      (g_base == nullptr || aligned16(g_base));
+    KernelScope scope(ctx, SAMA_K_ADAPT, -1, st);
     if (vec) {
         const int grid = stream_grid(ctx, n >> 2, kUnroll);
         if (g_base)
@@ -303,16 +304,15 @@ cudaError_t launch_adapt_sumsq(sama_ctx* ctx, int64_t n, const float* m, const f
             adapt_sumsq_scalar<false><<<grid, kThreads, 0, st>>>(n, m, s, nullptr, g_meta, p_out, c,
                                                                  ctx->partials, ctx->scalars, sumsq_out);
     }
-    ctx->launches += 1;
     return cudaGetLastError();
 }
 
 cudaError_t launch_sumsq(sama_ctx* ctx, int64_t n, const float* p, cudaStream_t st) {
+    KernelScope scope(ctx, SAMA_K_SUMSQ, -1, st);
     if (aligned16(p))
         sumsq_kernel<true><<<stream_grid(ctx, n >> 2, 4), kThreads, 0, st>>>(n, p, ctx->partials, ctx->scalars);
     else
         sumsq_kernel<false><<<stream_grid(ctx, n, 8), kThreads, 0, st>>>(n, p, ctx->partials, ctx->scalars);
-    ctx->launches += 1;
     return cudaGetLastError();
 }
 
@@ -320,13 +320,13 @@ cudaError_t launch_perturb(sama_ctx* ctx, int64_t n, const float* theta, const f
                            float alpha, float* theta_plus, float* theta_minus, float* eps_fd_out,
                            cudaStream_t st) {
     const bool vec = aligned16(theta) && aligned16(p) && aligned16(theta_plus) && aligned16(theta_minus);
+    KernelScope scope(ctx, SAMA_K_PERTURB, -1, st);
     if (vec)
         perturb_kernel<true><<<stream_grid(ctx, n >> 2, kUnroll), kThreads, 0, st>>>(
             n, theta, p, sumsq, alpha, theta_plus, theta_minus, ctx->scalars, eps_fd_out);
     else
         perturb_kernel<false><<<stream_grid(ctx, n, 4), kThreads, 0, st>>>(
             n, theta, p, sumsq, alpha, theta_plus, theta_minus, ctx->scalars, eps_fd_out);
-    ctx->launches += 1;
     return cudaGetLastError();
 }
 

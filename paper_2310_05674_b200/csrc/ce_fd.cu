@@ -69,9 +69,9 @@ cudaError_t launch_ce_fd(sama_ctx* ctx, const float* z_plus, const float* z_minu
                          const float* lambda, int B, int C, const float* eps_fd, float* metagrad,
                          float* loss_plus, float* loss_minus, cudaStream_t st) {
     const int grid = (B + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    KernelScope scope(ctx, SAMA_K_CE_FD, -1, st);
     ce_fd_kernel<<<grid, kWarpsPerBlock * 32, 0, st>>>(z_plus, z_minus, ldz, y, lambda, B, C, eps_fd, metagrad,
                                                        loss_plus, loss_minus, ctx->scalars);
-    ctx->launches += 1;
     return cudaGetLastError();
 }
 

@@ -178,7 +178,7 @@ cudaError_t launch_gemm_ffma(sama_ctx* ctx, const GemmArgs& g, cudaStream_t st) 
     auto ctas = [&](int bm, int bn) {
         return (int64_t)((g.M + bm - 1) / bm) * ((g.N + bn - 1) / bn) * 2;
     };
-    ctx->launches += 1;
+    KernelScope scope(ctx, SAMA_K_GEMM_FFMA, g.layer, st);
     // Largest tile that still gives every SM work; small problems take small tiles.
     if (ctas(128, 128) >= ctx->sm_count) return launch_variant<128, 128, 8, 8>(g, vec, st);
     if (ctas(64, 64) >= ctx->sm_count) return launch_variant<64, 64, 4, 4>(g, vec, st);

@@ -175,6 +175,7 @@ int run_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const 
         g.ldw = din;
         g.ldc = dout;
         g.relu = last ? 0 : 1;
+        g.layer = l;
         SAMA_CUDA(ctx, launch_gemm(ctx, g, st));
         in[0] = g.C[0];
         in[1] = g.C[1];
@@ -262,6 +263,10 @@ int sama_destroy(sama_ctx* ctx) {
     cudaFree(ctx->act[1]);
     cudaFree(ctx->logits);
     cudaFree(ctx->stage);
+    if (ctx->prof) {
+        for (auto& r : ctx->prof->records) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
+        delete ctx->prof;
+    }
     delete ctx;
     return SAMA_OK;
 }
@@ -437,6 +442,41 @@ int sama_set_gemm_mode(sama_ctx* ctx, int mode) {
 }
 
 int64_t sama_launch_count(sama_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int sama_profile_enable(sama_ctx* ctx, int32_t on) {
+    if (!ctx) return SAMA_ERR_NULL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SAMA_ERR_CUDA;
+    if (!ctx->prof) {
+        ctx->prof = new (std::nothrow) Profiler();
+        if (!ctx->prof) return SAMA_ERR_NOMEM;
+    }
+    for (auto& r : ctx->prof->records) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
+    ctx->prof->records.clear();
+    ctx->prof->on = (on != 0);
+    return SAMA_OK;
+}
+
+int sama_profile_collect(sama_ctx* ctx, sama_kernel_time_t* out, int32_t capacity, int32_t* count_out) {
+    if (!ctx || !count_out || (capacity > 0 && !out)) return SAMA_ERR_NULL;
+    *count_out = 0;
+    if (!ctx->prof) return SAMA_OK;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SAMA_ERR_CUDA;
+    int32_t k = 0;
+    for (auto& r : ctx->prof->records) {
+        float ms = 0.f;
+        cudaError_t e = cudaEventSynchronize(r.stop);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, r.start, r.stop);
+        cudaEventDestroy(r.start);
+        cudaEventDestroy(r.stop);
+        if (e != cudaSuccess) { ctx->prof->records.clear(); return cuda_fail(ctx, e); }
+        if (k < capacity) { out[k].kind = r.kind; out[k].layer = r.layer; out[k].ms = ms; ++k; }
+    }
+    ctx->prof->records.clear();
+    *count_out = k;
+    return SAMA_OK;
+}
 
 const char* sama_status_string(int status) {
     switch (status) {

@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "sama.h"
 
 namespace sama {
@@ -31,6 +33,15 @@ struct AdaptConsts {
     int identity;
 };
 
+struct ProfRecord {
+    int kind, layer;
+    cudaEvent_t start, stop;
+};
+struct Profiler {
+    bool on = false;
+    std::vector<ProfRecord> records;
+};
+
 }  // namespace sama
 
 struct sama_ctx {
@@ -49,9 +60,31 @@ struct sama_ctx {
     float* logits;                 // device [2][max_batch][max_classes]
     float* stage;                  // device: staging of the host entry point (allocated on first use)
     size_t stage_bytes;
+    sama::Profiler* prof;          // host
 };
 
 namespace sama {
+
+// Counts a launch and, while profiling is on, brackets it with two events on its stream.
+struct KernelScope {
+    sama_ctx* ctx;
+    cudaStream_t st;
+    cudaEvent_t stop = nullptr;
+    KernelScope(sama_ctx* c, int kind, int layer, cudaStream_t s) : ctx(c), st(s) {
+        ctx->launches += 1;
+        if (ctx->prof && ctx->prof->on) {
+            ProfRecord r{kind, layer, nullptr, nullptr};
+            if (cudaEventCreate(&r.start) == cudaSuccess && cudaEventCreate(&r.stop) == cudaSuccess) {
+                cudaEventRecord(r.start, st);
+                stop = r.stop;
+                ctx->prof->records.push_back(r);
+            }
+        }
+    }
+    ~KernelScope() {
+        if (stop) cudaEventRecord(stop, st);
+    }
+};
 
 // adapt_perturb.cu
 cudaError_t launch_adapt_sumsq(sama_ctx* ctx, int64_t n, const float* m, const float* s, const float* g_base,
@@ -70,6 +103,7 @@ struct GemmArgs {
     int M, N, K;
     int lda, ldw, ldc;
     int relu;
+    int layer;
 };
 // gemm_ffma.cu
 cudaError_t launch_gemm_ffma(sama_ctx* ctx, const GemmArgs& g, cudaStream_t st);

@@ -1,0 +1,366 @@
+"""GPU parity: the C-ABI CUDA path against the CPU checker, element by element,
+on the same seeded inputs.
+
+Tolerances (stated by the task this library was built for, restated here):
+  adaptation / perturbation : relative 1e-5 elementwise, eps_fd relative 1e-6;
+  FD meta-gradient          : |a-b| <= max(2e-3 |b|, 1e-6) elementwise, plus the
+                              same 2e-3 on the whole vector in the 2-norm.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2310_05674_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+from gpu_util import (B, Ctx, DEV, assert_adapt_close, assert_fd_close, dev, fd_errors, read_f32, read_f64,  # noqa: E402
+                      run_adapt, run_step, unaligned)
+
+
+def o_adam(a: "B.Adam") -> oracle.Adam:
+    return oracle.Adam(a.lr, a.beta1, a.beta2, a.eps, a.step, a.bias_correction, a.drop_eps_term, a.identity)
+
+
+ADAMS = {
+    "default": B.Adam(),
+    "step1": B.Adam(step=1),
+    "step1000": B.Adam(step=1000),
+    "nobias": B.Adam(bias_correction=False),
+    "dropeps": B.Adam(drop_eps_term=True),
+    "identity": B.Adam(identity=True),
+    "odd": B.Adam(lr=3e-2, beta1=0.8, beta2=0.99, eps=1e-6, step=7),
+}
+
+
+# ---------------------------------------------------------------- adapt ----
+
+@pytest.mark.parametrize("n", [0, 1, 3, 4, 5, 1023, 1025, 2 ** 20 + 1])
+@pytest.mark.parametrize("mode", sorted(ADAMS))
+def test_adapt_parity(n, mode):
+    adam = ADAMS[mode]
+    w = W.flat_vector(n, seed=n + 1)
+    ref = oracle.adapt(w["m"], w["s"], w["g_base"], w["g_meta"], o_adam(adam))
+    with Ctx(max(n, 1)) as ctx:
+        p, ss, _, _ = run_adapt(ctx, w, adam)
+        assert_adapt_close(p, ref)
+        if mode == "identity":
+            assert np.array_equal(p, w["g_meta"])
+        assert ss == pytest.approx(float(np.dot(p.astype(np.float64), p.astype(np.float64))), rel=1e-12, abs=1e-300)
+        assert ss == pytest.approx(oracle.sumsq(ref), rel=2e-6, abs=1e-300)
+        assert read_f64(B.sama_ctx_sumsq(ctx.h)) == ss
+
+
+@pytest.mark.parametrize("n", [5, 1025, 300001])
+def test_adapt_variants(n):
+    adam = B.Adam()
+    w = W.flat_vector(n, seed=77)
+    with Ctx(n) as ctx:
+        base, ss0, _, _ = run_adapt(ctx, w, adam)
+        # g_base = NULL means g := m
+        ref = oracle.adapt(w["m"], w["s"], None, w["g_meta"], o_adam(adam))
+        p, _, _, _ = run_adapt(ctx, w, adam, use_gbase=False)
+        assert_adapt_close(p, ref)
+        # unaligned pointers take the scalar kernels
+        full = oracle.adapt(w["m"], w["s"], w["g_base"], w["g_meta"], o_adam(adam))
+        for shift in (1, 3):
+            p, ss, _, _ = run_adapt(ctx, w, adam, shift=shift)
+            assert_adapt_close(p, full)
+            assert ss == pytest.approx(ss0, rel=1e-6)
+        # in place over g_meta
+        p, ss, _, _ = run_adapt(ctx, w, adam, inplace=True)
+        assert np.array_equal(p, base) and ss == ss0
+        # repeated calls are bit-identical (fixed reduction order)
+        p2, ss2, _, _ = run_adapt(ctx, w, adam)
+        assert np.array_equal(p2, base) and ss2 == ss0
+
+
+# -------------------------------------------------------------- perturb ----
+
+@pytest.mark.parametrize("n", [1, 3, 4, 1023, 1025, 2 ** 20 + 1])
+def test_perturb_parity(n):
+    w = W.flat_vector(n, seed=n + 5)
+    adam, alpha = B.Adam(), 0.37
+    with Ctx(n) as ctx:
+        p_np, ss, p_dev, ss_dev = run_adapt(ctx, w, adam)
+        rtp, rtm, reps, bad = oracle.perturb(w["theta"], p_np, alpha)
+        assert not bad
+        theta = dev(w["theta"])
+        tp, tm = torch.empty_like(theta), torch.empty_like(theta)
+        eps = torch.zeros(1, dtype=torch.float32, device=DEV)
+        B.sama_perturb(ctx.h, n, theta, p_dev, ss_dev, alpha, tp, tm, eps)
+        torch.cuda.synchronize()
+        assert float(eps.item()) == pytest.approx(reps, rel=1e-6)
+        assert read_f32(B.sama_ctx_eps_fd(ctx.h)) == float(eps.item())
+        assert_adapt_close(tp.cpu().numpy(), rtp, "theta_plus")
+        assert_adapt_close(tm.cpu().numpy(), rtm, "theta_minus")
+        # the displacement itself, not just theta + small: (theta+ - theta-)/2 = eps p to fp32 rounding of theta
+        d = (tp.double() - tm.double()).cpu().numpy() / 2
+        ulp = np.abs(w["theta"]).astype(np.float64) * 2.0 ** -23
+        assert np.all(np.abs(d - reps * p_np.astype(np.float64)) <= 1e-5 * np.abs(reps * p_np) + ulp)
+        # norm computed inside (p_sumsq = NULL) gives the same result
+        tp2, tm2 = torch.empty_like(theta), torch.empty_like(theta)
+        B.sama_perturb(ctx.h, n, theta, p_dev, None, alpha, tp2, tm2, None)
+        torch.cuda.synchronize()
+        assert read_f32(B.sama_ctx_eps_fd(ctx.h)) == pytest.approx(float(eps.item()), rel=1e-6)
+        assert_adapt_close(tp2.cpu().numpy(), rtp)
+        # theta_minus aliasing theta: the base-parameter nudge
+        th2 = theta.clone()
+        B.sama_perturb(ctx.h, n, th2, p_dev, ss_dev, alpha, tp2, th2, None)
+        torch.cuda.synchronize()
+        assert torch.equal(th2, tm) and torch.equal(tp2, tp)
+        # unaligned
+        thu, tpu, tmu = unaligned(w["theta"], 1), unaligned(np.zeros(n, np.float32), 1), unaligned(np.zeros(n, np.float32), 1)
+        B.sama_perturb(ctx.h, n, thu, p_dev, ss_dev, alpha, tpu, tmu, None)
+        torch.cuda.synchronize()
+        assert torch.equal(tpu, tp) and torch.equal(tmu, tm)
+        assert B.sama_device_status(ctx.h) == 0
+
+
+def test_perturb_degenerate_norm_sets_status():
+    n = 1000
+    with Ctx(n) as ctx:
+        theta = dev(W.flat_vector(n, 3)["theta"])
+        for bad_p in (np.zeros(n, np.float32), np.full(n, np.nan, np.float32), np.full(n, 3e38, np.float32).astype(np.float32) * np.float32(1e30)):
+            p = dev(bad_p.astype(np.float32))
+            tp, tm = torch.empty_like(theta), torch.empty_like(theta)
+            eps = torch.ones(1, dtype=torch.float32, device=DEV)
+            B.sama_perturb(ctx.h, n, theta, p, None, 1.0, tp, tm, eps)
+            assert B.sama_device_status(ctx.h) == B.SAMA_DEV_DEGENERATE_NORM
+            assert float(eps.item()) == 0.0
+            assert torch.equal(tp, theta) and torch.equal(tm, theta)
+        assert B.sama_device_status(ctx.h) == 0  # reading clears
+
+
+# ---------------------------------------------------- forward + FD alone ----
+
+RAGGED = [((12, 5), 1), ((33, 17, 12, 6), 7), ((100, 50, 3), 129), ((257, 130, 66, 11), 65), ((64, 64, 64, 16), 300)]
+
+
+@pytest.mark.parametrize("dims,batch", RAGGED)
+def test_fd_metagrad_parity_ragged(dims, batch):
+    cfg, w = W.custom_mlp(dims, batch, seed=sum(dims))
+    n = cfg.n_params
+    # non-zero biases and a realistic pair theta+-
+    theta = (w["theta"] + 0.05 * W.normal(5, 99, n).astype(np.float32)).astype(np.float32)
+    d = (1e-3 * W.normal(6, 98, n)).astype(np.float32)
+    tp_np, tm_np = (theta + d).astype(np.float32), (theta - d).astype(np.float32)
+    eps_val = np.float32(0.05)
+    lp = oracle.losses(dims, tp_np, w["X"], w["y"])
+    lm = oracle.losses(dims, tm_np, w["X"], w["y"])
+    ref = oracle.fd(lp, lm, w["lam"], float(eps_val), batch)
+    with Ctx(n, batch, dims) as ctx:
+        out = [torch.empty(batch, dtype=torch.float32, device=DEV) for _ in range(3)]
+        B.sama_fd_metagrad(ctx.h, ctx.mlp, dev(tp_np), dev(tm_np), dev(w["X"]), dev(w["y"]), dev(w["lam"]), batch,
+                           dev(np.array([eps_val])), out[0], out[1], out[2])
+        torch.cuda.synchronize()
+        np.testing.assert_allclose(out[1].cpu().numpy(), lp, rtol=2e-5, atol=2e-5)
+        np.testing.assert_allclose(out[2].cpu().numpy(), lm, rtol=2e-5, atol=2e-5)
+        assert_fd_close(out[0].cpu().numpy(), ref)
+        # the loss outputs are optional
+        mg2 = torch.empty(batch, dtype=torch.float32, device=DEV)
+        B.sama_fd_metagrad(ctx.h, ctx.mlp, dev(tp_np), dev(tm_np), dev(w["X"]), dev(w["y"]), dev(w["lam"]), batch,
+                           dev(np.array([eps_val])), mg2, None, None)
+        torch.cuda.synchronize()
+        assert torch.equal(mg2, out[0])
+        assert B.sama_device_status(ctx.h) == 0
+
+
+def test_bad_label_is_reported_not_faulted():
+    dims, batch = (20, 9, 4), 10
+    cfg, w = W.custom_mlp(dims, batch, seed=4)
+    y = w["y"].copy()
+    y[3], y[7] = 4, -1
+    with Ctx(cfg.n_params, batch, dims) as ctx:
+        mg = torch.empty(batch, dtype=torch.float32, device=DEV)
+        th = dev(w["theta"])
+        B.sama_fd_metagrad(ctx.h, ctx.mlp, th, dev(w["theta"] * np.float32(1.01)), dev(w["X"]), dev(y),
+                           dev(w["lam"]), batch, dev(np.float32([0.1])), mg, None, None)
+        assert B.sama_device_status(ctx.h) == B.SAMA_DEV_BAD_LABEL
+        mg = mg.cpu().numpy()
+        assert mg[3] == 0 and mg[7] == 0 and np.all(mg[[0, 1, 2, 4, 5, 6, 8, 9]] != 0)
+
+
+# ------------------------------------------------------------ whole step ----
+
+def check_step(cfg, w, adam, alpha, rows=None, use_gbase=True):
+    """Runs sama_step on the full batch; the checker runs on ``rows`` (all if None)."""
+    with Ctx(cfg.n_params, cfg.batch, cfg.dims) as ctx:
+        got = run_step(ctx, cfg, w, adam, alpha, use_gbase=use_gbase)
+    sel = slice(None) if rows is None else rows
+    ref = oracle.step(cfg.dims, w["theta"], w["m"], w["s"], w["g_base"] if use_gbase else None, w["g_meta"],
+                      o_adam(adam), alpha, w["X"][sel], w["y"][sel], w["lam"][sel], B_norm=cfg.batch)
+    assert got["status"] == 0 and not ref["degenerate"]
+    assert_adapt_close(got["p"], ref["p"])
+    assert got["eps_fd"] == pytest.approx(ref["eps_fd"], rel=1e-6)
+    assert_adapt_close(got["theta_plus"], ref["theta_plus"], "theta_plus")
+    assert_adapt_close(got["theta_minus"], ref["theta_minus"], "theta_minus")
+    np.testing.assert_allclose(got["loss_plus"][sel], ref["loss_plus"], rtol=1e-4, atol=1e-4)
+    e = assert_fd_close(got["metagrad"][sel], ref["metagrad"])
+    # the per-sample difference quotient before the sigmoid'/B scaling, same 2e-3 in the 2-norm
+    dq = (got["loss_plus"].astype(np.float64) - got["loss_minus"].astype(np.float64))[sel]
+    dr = ref["loss_plus"] - ref["loss_minus"]
+    e["dq_norm_rel"] = float(np.linalg.norm(dq - dr) / np.linalg.norm(dr))
+    print("\n[parity] %s alpha=%g: %s" % (cfg.name, alpha, e))
+    return e
+
+
+@pytest.mark.parametrize("alpha", [1e-2, 1.0])
+def test_step_parity_tiny(alpha):
+    cfg = W.CONFIGS["tiny"]
+    check_step(cfg, W.mlp_workload(cfg, 0), B.Adam(), alpha)
+
+
+def test_step_parity_tiny_variants():
+    cfg = W.CONFIGS["tiny"]
+    w = W.mlp_workload(cfg, 0)
+    check_step(cfg, w, B.Adam(), 1e-2, use_gbase=False)
+    check_step(cfg, w, B.Adam(identity=True), 1e-2)
+    check_step(cfg, w, B.Adam(step=1, drop_eps_term=True), 1e-2)
+
+
+@pytest.mark.parametrize("dims,batch", RAGGED[1:])
+def test_step_parity_ragged(dims, batch):
+    cfg, w = W.custom_mlp(dims, batch, seed=3 + sum(dims))
+    check_step(cfg, w, B.Adam(), 1e-2)
+
+
+def test_step_parity_mlp3072():
+    cfg = W.CONFIGS["mlp3072"]
+    w = W.mlp_workload(cfg, 0)
+    check_step(cfg, w, B.Adam(), 1e-2)
+    check_step(cfg, w, B.Adam(), 1.0, rows=np.arange(0, cfg.batch, 8))
+
+
+def test_step_parity_head1024():
+    cfg = W.CONFIGS["head1024"]
+    w = W.mlp_workload(cfg, 0)
+    check_step(cfg, w, B.Adam(), 1e-2)
+    check_step(cfg, w, B.Adam(), 1.0, rows=np.arange(0, cfg.batch, 64))
+
+
+def test_step_parity_wide4096_sampled():
+    """Full-size launch; the checker evaluates a sample of the rows (each output
+    depends only on its own row given theta+-, which are compared in full)."""
+    cfg = W.CONFIGS["wide4096"]
+    w = W.mlp_workload(cfg, 0)
+    rows = np.unique(np.concatenate([np.arange(0, cfg.batch, 97), [cfg.batch - 1]]))
+    check_step(cfg, w, B.Adam(), 1e-2, rows=rows)
+
+
+def test_step_host_matches_step():
+    cfg = W.CONFIGS["tiny"]
+    w = W.mlp_workload(cfg, 0)
+    adam, alpha = B.Adam(), 1e-2
+    with Ctx(cfg.n_params, cfg.batch, cfg.dims) as ctx:
+        got = run_step(ctx, cfg, w, adam, alpha)
+        pin = {k: torch.from_numpy(np.ascontiguousarray(w[k])).pin_memory()
+               for k in ["theta", "m", "s", "g_base", "g_meta", "X", "y", "lam"]}
+        mg = torch.empty(cfg.batch, dtype=torch.float32).pin_memory()
+        eps = torch.empty(1, dtype=torch.float32).pin_memory()
+        tm = torch.empty(cfg.n_params, dtype=torch.float32).pin_memory()
+        B.sama_step_host(ctx.h, ctx.mlp, cfg.n_params, pin["theta"], pin["m"], pin["s"], pin["g_base"],
+                         pin["g_meta"], adam, alpha, pin["X"], pin["y"], pin["lam"], cfg.batch, mg, eps, tm)
+        assert np.array_equal(mg.numpy(), got["metagrad"])
+        assert float(eps.item()) == got["eps_fd"]
+        assert np.array_equal(tm.numpy(), got["theta_minus"])
+
+
+# ------------------------------------------------ flat vectors, full size ----
+
+@pytest.mark.parametrize("name", ["flat110m", "flat355m"])
+def test_flat_vector_full_size(name):
+    """adapt + norm + perturb on BERT-base / RoBERTa-large sized vectors, every
+    element compared; the checker runs in slices to bound host memory."""
+    n = W.FLAT_SIZES[name]
+    w = W.flat_vector(n, seed=0)
+    alpha = 1.0
+    t = {k: dev(w[k]) for k in ["theta", "m", "s", "g_base", "g_meta"]}
+    p, tp, tm = (torch.empty(n, dtype=torch.float32, device=DEV) for _ in range(3))
+    chunk = 1 << 24
+    with Ctx(n) as ctx:
+        for step in (1, 1000):
+            adam = B.Adam(step=step)
+            B.sama_adapt(ctx.h, n, t["m"], t["s"], t["g_base"], t["g_meta"], adam, p, None)
+            B.sama_perturb(ctx.h, n, t["theta"], p, B.sama_ctx_sumsq(ctx.h), alpha, tp, tm, None)
+            torch.cuda.synchronize()
+            assert B.sama_device_status(ctx.h) == 0
+            gp, gtp, gtm = p.cpu().numpy(), tp.cpu().numpy(), tm.cpu().numpy()
+            refs, total = [], 0.0
+            for a in range(0, n, chunk):
+                b = min(n, a + chunk)
+                rp = oracle.adapt(w["m"][a:b], w["s"][a:b], w["g_base"][a:b], w["g_meta"][a:b], o_adam(adam))
+                total += oracle.sumsq(rp)
+                refs.append(rp)
+            assert read_f64(B.sama_ctx_sumsq(ctx.h)) == pytest.approx(total, rel=2e-6)
+            pmax = max(float(np.abs(r).max()) for r in refs)
+            worst = 0.0
+            eps_ref = None
+            for i, a in enumerate(range(0, n, chunk)):
+                b = min(n, a + chunk)
+                rp = refs[i]
+                scale = np.maximum(np.abs(rp), 1e-3 * pmax)
+                worst = max(worst, float((np.abs(gp[a:b] - rp) / scale).max()))
+                rtp, rtm, eps_ref, bad = oracle.perturb_given_sumsq(w["theta"][a:b], rp, total, alpha)
+                assert not bad
+                for g_, r_ in ((gtp[a:b], rtp), (gtm[a:b], rtm)):
+                    assert float((np.abs(g_ - r_) / np.maximum(np.abs(r_), 1e-4)).max()) <= 1e-5
+            assert worst <= 1e-5, worst
+            assert read_f32(B.sama_ctx_eps_fd(ctx.h)) == pytest.approx(eps_ref, rel=1e-6)
+            print("\n[parity] %s step=%d: max rel err p %.3e" % (name, step, worst))
+
+
+# ---------------------------------------------------------- error paths ----
+
+def test_argument_errors_are_caught_on_the_host():
+    n = 64
+    cfg, w = W.custom_mlp((8, 4, 3), 5, seed=1)
+    with Ctx(n, 5, (8, 4, 3)) as ctx:
+        buf = torch.zeros(8 * n, dtype=torch.float32, device=DEV)
+        a = [buf[i * n:(i + 1) * n] for i in range(8)]
+        adam = B.Adam()
+
+        def status(fn, *args, **kw):
+            with pytest.raises(B.SamaError) as e:
+                fn(*args, **kw)
+            return e.value.status
+
+        assert status(B.sama_adapt, ctx.h, n, None, a[1], None, a[2], adam, a[3]) == B.SAMA_ERR_NULL
+        assert status(B.sama_adapt, ctx.h, n, a[0], a[1], None, None, adam, a[3]) == B.SAMA_ERR_NULL
+        assert status(B.sama_adapt, ctx.h, -1, a[0], a[1], None, a[2], adam, a[3]) == B.SAMA_ERR_SIZE
+        assert status(B.sama_adapt, ctx.h, n + 1, a[0], a[1], None, a[2], adam, a[3]) == B.SAMA_ERR_SIZE
+        assert status(B.sama_adapt, ctx.h, n, a[0].data_ptr() + 2, a[1], None, a[2], adam, a[3]) == B.SAMA_ERR_ALIGN
+        assert status(B.sama_adapt, ctx.h, n, a[0], a[1], None, a[2], adam, a[0]) == B.SAMA_ERR_OVERLAP
+        assert status(B.sama_adapt, ctx.h, n, a[0], a[1], None, a[2], adam, a[2].data_ptr() + 16) == B.SAMA_ERR_OVERLAP
+        for bad in (B.Adam(step=0), B.Adam(beta1=1.0), B.Adam(beta2=-0.1), B.Adam(lr=float("nan")),
+                    B.Adam(lr=0.0), B.Adam(eps=float("inf")), B.Adam(eps=-1e-8)):
+            assert status(B.sama_adapt, ctx.h, n, a[0], a[1], None, a[2], bad, a[3]) == B.SAMA_ERR_PARAM
+        # identity mode needs neither moments nor valid Adam scalars
+        assert B.sama_adapt(ctx.h, n, None, None, None, a[2], B.Adam(identity=True, lr=float("nan")), a[3]) == 0
+
+        assert status(B.sama_perturb, ctx.h, n, a[0], a[1], None, 0.0, a[2], a[3]) == B.SAMA_ERR_PARAM
+        assert status(B.sama_perturb, ctx.h, n, a[0], a[1], None, float("inf"), a[2], a[3]) == B.SAMA_ERR_PARAM
+        assert status(B.sama_perturb, ctx.h, n, a[0], a[1], None, 1.0, a[2], a[2]) == B.SAMA_ERR_OVERLAP
+        assert status(B.sama_perturb, ctx.h, n, a[0], a[1], None, 1.0, a[0], a[3]) == B.SAMA_ERR_OVERLAP
+        assert status(B.sama_perturb, ctx.h, n, a[0], a[1], None, 1.0, a[2], a[1]) == B.SAMA_ERR_OVERLAP
+        assert status(B.sama_perturb, ctx.h, n, a[0], None, None, 1.0, a[2], a[3]) == B.SAMA_ERR_NULL
+
+        mlp = ctx.mlp
+        X, y, lam = dev(w["X"]), dev(w["y"]), dev(w["lam"])
+        mg = torch.zeros(5, dtype=torch.float32, device=DEV)
+        eps = torch.ones(1, dtype=torch.float32, device=DEV)
+        assert status(B.sama_fd_metagrad, ctx.h, mlp, a[0], a[1], X, y, lam, 0, eps, mg) == B.SAMA_ERR_SIZE
+        assert status(B.sama_fd_metagrad, ctx.h, mlp, a[0], a[1], X, y, lam, 6, eps, mg) == B.SAMA_ERR_SIZE
+        assert status(B.sama_fd_metagrad, ctx.h, B.MLP((8, 5, 3)), a[0], a[1], X, y, lam, 5, eps, mg) == B.SAMA_ERR_SIZE
+        assert status(B.sama_fd_metagrad, ctx.h, B.MLP((8, 4, 4)), a[0], a[1], X, y, lam, 5, eps, mg) == B.SAMA_ERR_SIZE
+        assert status(B.sama_fd_metagrad, ctx.h, mlp, a[0], a[1], X, None, lam, 5, eps, mg) == B.SAMA_ERR_NULL
+        assert status(B.sama_fd_metagrad, ctx.h, mlp, a[0], a[1], X, y, lam, 5, eps, lam) == B.SAMA_ERR_OVERLAP
+        # n must be the model's parameter count
+        assert status(B.sama_step, ctx.h, mlp, n, a[0], a[1], a[2], None, a[3], adam, 1.0, X, y, lam, 5,
+                      a[4], a[5], a[6], mg) == B.SAMA_ERR_SIZE
+        assert B.sama_last_cuda_error(ctx.h) == 0
+        assert B.sama_device_status(ctx.h) == 0
+    # a context without a model cannot run the forward pass
+    with Ctx(n) as ctx:
+        assert status(B.sama_fd_metagrad, ctx.h, B.MLP((8, 4, 3)), a[0], a[1], X, y, lam, 5, eps, mg) == B.SAMA_ERR_SIZE
