@@ -125,42 +125,58 @@ def recorded_traffic(kernel: str, workload: str):
     return None
 
 
-def oracle_step_seconds(cfg, w, budget_s=15.0):
-    """Times the CPU checker as it stands on a bounded sample of the workload and
-    scales to a whole step.  Returns (seconds per full step, description, rows used)."""
-    import oracle
-    adam = oracle.Adam()
-    B = cfg.batch
-    t0 = time.perf_counter()
-    oracle.step(cfg.dims, w["theta"], w["m"], w["s"], w["g_base"], w["g_meta"], adam, cfg.alpha,
-                w["X"][:1], w["y"][:1], w["lam"][:1], B_norm=B)
-    t1 = time.perf_counter() - t0          # elementwise stages over all n + one row of forward
-    t0 = time.perf_counter()
-    p = oracle.adapt(w["m"], w["s"], w["g_base"], w["g_meta"], adam)
-    oracle.perturb(w["theta"], p, cfg.alpha)
-    t_elem = time.perf_counter() - t0
-    per_row = max(t1 - t_elem, 1e-6)
-    rows = int(max(1, min(B, budget_s / per_row)))
-    t0 = time.perf_counter()
-    oracle.step(cfg.dims, w["theta"], w["m"], w["s"], w["g_base"], w["g_meta"], adam, cfg.alpha,
-                w["X"][:rows], w["y"][:rows], w["lam"][:rows], B_norm=B)
-    t_rows = time.perf_counter() - t0
-    fwd = max(t_rows - t_elem, 1e-9)
-    full = t_elem + fwd * (B / rows)
-    desc = ("adapt+norm+perturb over all %d parameters, forward+FD on rows 0..%d of %d with the forward "
-            "time scaled by %d/%d" % (cfg.n_params, rows - 1, B, B, rows))
-    return full, desc, rows
+class OracleTimer:
+    """Times the CPU checker, as it stands, on a bounded sample of the workload:
+    the elementwise stages on the first `cnt` of n parameters and the forward +
+    finite difference on the first `rows` of B samples, each scaled to the whole
+    workload.  theta+- for the forward are prepared once, outside the timing."""
 
+    def __init__(self, name, w, cfg):
+        import oracle
+        self.o, self.name, self.w, self.cfg = oracle, name, w, cfg
+        self.n = w["theta"].size
+        self.adam = oracle.Adam(float(np.float32(1e-3)), float(np.float32(0.9)), float(np.float32(0.999)),
+                                float(np.float32(1e-8)), 100)
+        self.alpha = cfg.alpha if cfg else 1.0
+        self.elem_rate = None   # seconds per parameter
+        self.row_rate = None    # seconds per sample
+        if cfg:
+            p = oracle.adapt(w["m"], w["s"], w["g_base"], w["g_meta"], self.adam)
+            self.tp, self.tm, self.eps, _ = oracle.perturb(w["theta"], p, self.alpha)
 
-def oracle_flat_seconds(n, w):
-    import oracle
-    adam = oracle.Adam()
-    cnt = min(n, 1 << 24)
-    t0 = time.perf_counter()
-    p = oracle.adapt(w["m"][:cnt], w["s"][:cnt], w["g_base"][:cnt], w["g_meta"][:cnt], adam)
-    oracle.perturb(w["theta"][:cnt], p, 1.0)
-    t = time.perf_counter() - t0
-    return t * (n / cnt), "elements 0..%d of %d, time scaled by %d/%d" % (cnt - 1, n, n, cnt), cnt
+    def elementwise(self, cnt):
+        w, o = self.w, self.o
+        t0 = time.perf_counter()
+        p = o.adapt(w["m"][:cnt], w["s"][:cnt], w["g_base"][:cnt], w["g_meta"][:cnt], self.adam)
+        o.perturb(w["theta"][:cnt], p, self.alpha)
+        return time.perf_counter() - t0
+
+    def forward(self, rows):
+        w, o, cfg = self.w, self.o, self.cfg
+        t0 = time.perf_counter()
+        lp = o.losses(cfg.dims, self.tp, w["X"][:rows], w["y"][:rows])
+        lm = o.losses(cfg.dims, self.tm, w["X"][:rows], w["y"][:rows])
+        o.fd(lp, lm, w["lam"][:rows], self.eps, cfg.batch)
+        return time.perf_counter() - t0
+
+    def step_seconds(self, budget_s):
+        """One sampled step within about budget_s of CPU time -> (seconds for a whole step, description)."""
+        n = self.n
+        if self.elem_rate is None:
+            c0 = min(n, 1 << 16)
+            self.elem_rate = self.elementwise(c0) / c0
+            if self.cfg:
+                self.row_rate = self.forward(1)
+        share = budget_s / (2.0 if self.cfg else 1.0)
+        cnt = int(max(1, min(n, share / self.elem_rate)))
+        t = self.elementwise(cnt) * (n / cnt)
+        desc = "adapt+norm+perturb on parameters 0..%d of %d (time x %d/%d)" % (cnt - 1, n, n, cnt)
+        if self.cfg:
+            B = self.cfg.batch
+            rows = int(max(1, min(B, share / self.row_rate)))
+            t += self.forward(rows) * (B / rows)
+            desc += "; dual forward + FD on samples 0..%d of %d (time x %d/%d)" % (rows - 1, B, B, rows)
+        return t, desc
 
 
 def run_reference(args):
@@ -169,28 +185,24 @@ def run_reference(args):
         return
     name = args.workload
     flat = name in W.FLAT_SIZES
-    if flat:
-        n = W.FLAT_SIZES[name]
-        w = W.flat_vector(n, 0)
-    else:
-        cfg = W.CONFIGS[name]
-        w = W.mlp_workload(cfg, 0)
-    budget = max(2.0, 120.0 / max(1, args.steps + args.warmup))
+    cfg = None if flat else W.CONFIGS[name]
+    w = W.flat_vector(W.FLAT_SIZES[name], 0) if flat else W.mlp_workload(cfg, 0)
+    timer = OracleTimer(name, w, cfg)
+    budget = 150.0 / max(1, args.steps + args.warmup)
     times, desc = [], ""
     for i in range(args.warmup + args.steps):
-        if flat:
-            t, desc, _ = oracle_flat_seconds(n, w)
-        else:
-            t, desc, _ = oracle_step_seconds(cfg, w, budget_s=budget)
+        t, desc = timer.step_seconds(budget)
         if i >= args.warmup:
             times.append(t)
     sec = sum(times) / len(times)
     value = 1.0 / sec
-    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": args.gpus,
+    out = {"impl": "reference", "metric": METRIC if not flat else "adapt+perturb sweeps/sec", "value": value,
+           "unit": "steps/s", "n_gpus": args.gpus,
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
            "config": {"workload": name},
-           "cpu_baseline": {"value": value, "unit": "steps/s", "cores": 1, "kind": "oracle", "sample": desc},
+           "cpu_baseline": {"value": value, "unit": "steps/s", "cores": 1, "kind": "oracle",
+                            "sample": "each step: " + desc},
            "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(out), flush=True)
 
@@ -198,7 +210,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mlp3072", choices=sorted(W.CONFIGS) + sorted(W.FLAT_SIZES))
@@ -399,10 +411,7 @@ def main():
         out["adapt_perturb_gbs"] = 36.0 * n / (ms_per_step * 1e-3) / 1e9
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        if flat:
-            sec, desc, _ = oracle_flat_seconds(n, w)
-        else:
-            sec, desc, _ = oracle_step_seconds(cfg, w)
+        sec, desc = OracleTimer(name, w, cfg).step_seconds(20.0)
         out["cpu_baseline"] = {"value": 1.0 / sec, "unit": "steps/s", "cores": 1, "kind": "oracle", "sample": desc,
                                "host_cores_available": os.cpu_count()}
     S.sama_destroy(ctx)

@@ -20,7 +20,10 @@ from gpu_util import (B, Ctx, DEV, assert_adapt_close, assert_fd_close, dev, fd_
 
 
 def o_adam(a: "B.Adam") -> oracle.Adam:
-    return oracle.Adam(a.lr, a.beta1, a.beta2, a.eps, a.step, a.bias_correction, a.drop_eps_term, a.identity)
+    """The same hyper-parameters as the C ABI receives them: rounded to fp32."""
+    f = lambda x: float(np.float32(x))
+    return oracle.Adam(f(a.lr), f(a.beta1), f(a.beta2), f(a.eps), a.step, a.bias_correction, a.drop_eps_term,
+                       a.identity)
 
 
 ADAMS = {
