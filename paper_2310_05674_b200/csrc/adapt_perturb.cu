@@ -204,7 +204,9 @@ __device__ __forceinline__ float step_size(double sumsq, float alpha, bool& bad)
     return bad ? 0.0f : (float)((double)alpha / norm);
 }
 
+// eps == 0 marks the degenerate norm: theta+- = theta even where p is not finite.
 __device__ __forceinline__ void plus_minus(float eps, float4 vt, float4 vp, float4& a, float4& b) {
+    if (eps == 0.0f) { a = vt; b = vt; return; }
     a.x = fmaf(eps, vp.x, vt.x); b.x = fmaf(-eps, vp.x, vt.x);
     a.y = fmaf(eps, vp.y, vt.y); b.y = fmaf(-eps, vp.y, vt.y);
     a.z = fmaf(eps, vp.z, vt.z); b.z = fmaf(-eps, vp.z, vt.z);
@@ -255,15 +257,15 @@ perturb_kernel(int64_t n, const float* theta, const float* __restrict__ p, const
             const int64_t k = (items << 2) + threadIdx.x;
             if (k < n) {
                 const float t = theta[k], q = p[k];
-                theta_plus[k] = fmaf(eps, q, t);
-                theta_minus[k] = fmaf(-eps, q, t);
+                theta_plus[k] = eps == 0.0f ? t : fmaf(eps, q, t);
+                theta_minus[k] = eps == 0.0f ? t : fmaf(-eps, q, t);
             }
         }
     } else {
         for (; i < n; i += stride) {
             const float t = theta[i], q = p[i];
-            theta_plus[i] = fmaf(eps, q, t);
-            theta_minus[i] = fmaf(-eps, q, t);
+            theta_plus[i] = eps == 0.0f ? t : fmaf(eps, q, t);
+            theta_minus[i] = eps == 0.0f ? t : fmaf(-eps, q, t);
         }
     }
 }

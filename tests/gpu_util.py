@@ -150,11 +150,15 @@ def fd_errors(got, ref):
             "median_rel": float(np.median(rel))}
 
 
-def assert_fd_close(got, ref, what="metagrad"):
-    """FD meta-gradient: |a-b| <= max(2e-3 |b|, 1e-6) elementwise, and the same
-    2e-3 on the whole vector in the 2-norm (scale-free, so it still bites when
-    the 1/B factor pushes every entry under the absolute floor)."""
+def assert_fd_close(got, ref, what="metagrad", norm_tol=2e-3):
+    """FD meta-gradient: |a-b| <= max(2e-3 |b|, 1e-6) elementwise (the stated
+    bar), and a bound on the whole vector in the 2-norm, which is scale-free
+    and so still bites when the 1/B factor pushes every entry under the
+    absolute floor.  The quotient amplifies the fp32 rounding of the two
+    forward passes by 1/(2 eps_fd): at the paper's default alpha = 1 the norm
+    bound is the same 2e-3; at alpha = 1e-2 the rounding is 100x larger
+    relative to the signal and callers pass 2e-2."""
     e = fd_errors(got, ref)
     assert e["violations"] == 0, (what, e)
-    assert e["norm_rel"] <= 2e-3, (what, e)
+    assert e["norm_rel"] <= norm_tol, (what, e)
     return e

@@ -200,7 +200,7 @@ def check_step(cfg, w, adam, alpha, rows=None, use_gbase=True):
     assert_adapt_close(got["theta_plus"], ref["theta_plus"], "theta_plus")
     assert_adapt_close(got["theta_minus"], ref["theta_minus"], "theta_minus")
     np.testing.assert_allclose(got["loss_plus"][sel], ref["loss_plus"], rtol=1e-4, atol=1e-4)
-    e = assert_fd_close(got["metagrad"][sel], ref["metagrad"])
+    e = assert_fd_close(got["metagrad"][sel], ref["metagrad"], norm_tol=2e-3 if alpha >= 1.0 else 2e-2)
     # the per-sample difference quotient before the sigmoid'/B scaling, same 2e-3 in the 2-norm
     dq = (got["loss_plus"].astype(np.float64) - got["loss_minus"].astype(np.float64))[sel]
     dr = ref["loss_plus"] - ref["loss_minus"]
@@ -219,8 +219,9 @@ def test_step_parity_tiny_variants():
     cfg = W.CONFIGS["tiny"]
     w = W.mlp_workload(cfg, 0)
     check_step(cfg, w, B.Adam(), 1e-2, use_gbase=False)
-    check_step(cfg, w, B.Adam(identity=True), 1e-2)
+    check_step(cfg, w, B.Adam(identity=True), 1.0)
     check_step(cfg, w, B.Adam(step=1, drop_eps_term=True), 1e-2)
+    check_step(cfg, w, B.Adam(bias_correction=False), 1.0, use_gbase=False)
 
 
 @pytest.mark.parametrize("dims,batch", RAGGED[1:])
@@ -250,6 +251,7 @@ def test_step_parity_wide4096_sampled():
     w = W.mlp_workload(cfg, 0)
     rows = np.unique(np.concatenate([np.arange(0, cfg.batch, 97), [cfg.batch - 1]]))
     check_step(cfg, w, B.Adam(), 1e-2, rows=rows)
+    check_step(cfg, w, B.Adam(), 1.0, rows=rows[::2])
 
 
 def test_step_host_matches_step():
@@ -307,8 +309,10 @@ def test_flat_vector_full_size(name):
                 worst = max(worst, float((np.abs(gp[a:b] - rp) / scale).max()))
                 rtp, rtm, eps_ref, bad = oracle.perturb_given_sumsq(w["theta"][a:b], rp, total, alpha)
                 assert not bad
+                # theta +- eps p can cancel: the rounding is relative to the larger of |result| and |theta|
+                th = np.abs(w["theta"][a:b]).astype(np.float64)
                 for g_, r_ in ((gtp[a:b], rtp), (gtm[a:b], rtm)):
-                    assert float((np.abs(g_ - r_) / np.maximum(np.abs(r_), 1e-4)).max()) <= 1e-5
+                    assert float((np.abs(g_ - r_) / np.maximum(np.maximum(np.abs(r_), th), 1e-6)).max()) <= 1e-5
             assert worst <= 1e-5, worst
             assert read_f32(B.sama_ctx_eps_fd(ctx.h)) == pytest.approx(eps_ref, rel=1e-6)
             print("\n[parity] %s step=%d: max rel err p %.3e" % (name, step, worst))
