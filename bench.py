@@ -217,6 +217,7 @@ def main():
     ap.add_argument("--gemm-mode", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--flat-n", type=int, default=0, help="override the length of a flat-vector workload")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -254,7 +255,7 @@ def main():
     flat = name in W.FLAT_SIZES
     seed = rank  # each rank owns an independent batch / vector: no data-path collective
     if flat:
-        n = W.FLAT_SIZES[name]
+        n = args.flat_n or W.FLAT_SIZES[name]
         w = W.flat_vector(n, seed)
         cfg = None
         ctx = S.sama_create(local, n, 0, None)
