@@ -105,6 +105,36 @@ int sama_destroy(sama_ctx* ctx);
 int sama_adapt(sama_ctx* ctx, int64_t n, const float* m, const float* s, const float* g_base,
                const float* g_meta, const sama_adam_t* adam, float* p_out, double* sumsq_out, void* stream);
 
+/* sama_adapt without a context and without any allocation.  (The paper has no
+ * counterpart: this entry point exists for the deployment reason below.)
+ *
+ * sama_create allocates the reduction's scratch with cudaMalloc.  Callers that
+ * may not allocate -- code living under a framework whose caching allocator
+ * owns the device and forbids raw cudaMalloc, a plug-in loaded after a serving
+ * engine has sized and frozen its memory pools, initialisation paths where a
+ * synchronising allocation is not permitted -- use this instead: the scratch
+ * (one partial per block, an arrival counter; 33,024 bytes) is a static device
+ * array that every GPU loading the library holds until the process exits.
+ *
+ * Same arguments and results as sama_adapt, on the CURRENT device, except:
+ *   - sumsq_out (one double on the device) is required: there is no context
+ *     to leave the sum in;
+ *   - n may not exceed SAMA_NOALLOC_MAX_N; larger n returns SAMA_ERR_SIZE
+ *     before anything is launched (use sama_adapt with a context);
+ *   - the first call on each device resolves the array's device address
+ *     (cudaGetSymbolAddress) and reads the SM count; make that first call
+ *     outside any stream capture;
+ *   - every call on a device shares the one array.  It is cleared on the
+ *     stream at the start of each call, so calls issued one after another on
+ *     one stream are safe; calls that can overlap on the GPU (different
+ *     streams, no ordering) race on it and give wrong sums.
+ * Calls cudaGetDevice, cudaGetSymbolAddress / cudaDeviceGetAttribute (first
+ * call only), cudaMemsetAsync and one kernel launch; never cudaMalloc or
+ * cudaFree. */
+#define SAMA_NOALLOC_MAX_N ((int64_t)1 << 30)
+int sama_adapt_noalloc(int64_t n, const float* m, const float* s, const float* g_base, const float* g_meta,
+                       const sama_adam_t* adam, float* p_out, double* sumsq_out, void* stream);
+
 /* Sec. 3.2: eps_fd = alpha / sqrt(sumsq);  theta_plus = theta + eps_fd p,
  * theta_minus = theta - eps_fd p, written in one sweep.
  * p_sumsq: device double holding sum p^2 (e.g. sama_adapt's), or NULL to have

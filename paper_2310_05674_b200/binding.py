@@ -86,6 +86,7 @@ _vp = C.c_void_p
 lib.sama_create.argtypes = [C.POINTER(_vp), C.c_int, C.c_int64, C.c_int32, C.POINTER(sama_mlp_t)]
 lib.sama_destroy.argtypes = [_vp]
 lib.sama_adapt.argtypes = [_vp, C.c_int64, _vp, _vp, _vp, _vp, C.POINTER(sama_adam_t), _vp, _vp, _vp]
+lib.sama_adapt_noalloc.argtypes = [C.c_int64, _vp, _vp, _vp, _vp, C.POINTER(sama_adam_t), _vp, _vp, _vp]
 lib.sama_perturb.argtypes = [_vp, C.c_int64, _vp, _vp, _vp, C.c_float, _vp, _vp, _vp, _vp]
 lib.sama_fd_metagrad.argtypes = [_vp, C.POINTER(sama_mlp_t), _vp, _vp, _vp, _vp, _vp, C.c_int32, _vp, _vp, _vp,
                                  _vp, _vp]
@@ -157,6 +158,16 @@ def sama_adapt(ctx, n, m, s, g_base, g_meta, adam: Adam, p_out, sumsq_out=None, 
     a = adam.c()
     return _check(lib.sama_adapt(ctx, int(n), _ptr(m), _ptr(s), _ptr(g_base), _ptr(g_meta), C.byref(a),
                                  _ptr(p_out), _ptr(sumsq_out), _stream(stream)), "sama_adapt")
+
+
+SAMA_NOALLOC_MAX_N = 1 << 30
+
+
+def sama_adapt_noalloc(n, m, s, g_base, g_meta, adam: Adam, p_out, sumsq_out, stream=None) -> int:
+    """sama_adapt for callers that must not allocate: no context, static device scratch, current device."""
+    a = adam.c()
+    return _check(lib.sama_adapt_noalloc(int(n), _ptr(m), _ptr(s), _ptr(g_base), _ptr(g_meta), C.byref(a),
+                                         _ptr(p_out), _ptr(sumsq_out), _stream(stream)), "sama_adapt_noalloc")
 
 
 def sama_perturb(ctx, n, theta, p, p_sumsq, alpha, theta_plus, theta_minus, eps_fd_out=None, stream=None) -> int:

@@ -44,14 +44,9 @@ inline bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
     return x < y + nb && y < x + na;
 }
 
-int check_mlp(const sama_mlp_t* mlp) {
-    if (!mlp || !mlp->dims) return SAMA_ERR_NULL;
-    if (mlp->n_layers < 1 || mlp->n_layers > kMaxLayers) return SAMA_ERR_SIZE;
-    for (int l = 0; l <= mlp->n_layers; ++l)
-        if (mlp->dims[l] < 1) return SAMA_ERR_SIZE;
-    return SAMA_OK;
-}
+}  // namespace
 
+namespace sama {
 int check_adam(const sama_adam_t* a, AdaptConsts* out) {
     if (!a) return SAMA_ERR_NULL;
     AdaptConsts c;
@@ -81,14 +76,14 @@ int check_adam(const sama_adam_t* a, AdaptConsts* out) {
     return SAMA_OK;
 }
 
-int validate_adapt(sama_ctx* ctx, int64_t n, const float* m, const float* s, const float* g_base,
+int validate_adapt(int64_t max_n, int64_t n, const float* m, const float* s, const float* g_base,
                    const float* g_meta, const sama_adam_t* adam, float* p_out, double* sumsq_out,
                    AdaptConsts* c) {
-    if (!ctx || !adam || !g_meta || !p_out) return SAMA_ERR_NULL;
+    if (!adam || !g_meta || !p_out) return SAMA_ERR_NULL;
     const int rc = check_adam(adam, c);
     if (rc != SAMA_OK) return rc;
     if (!c->identity && (!m || !s)) return SAMA_ERR_NULL;
-    if (n < 0 || n > ctx->max_n) return SAMA_ERR_SIZE;
+    if (n < 0 || n > max_n) return SAMA_ERR_SIZE;
     if (!aligned(m, 4) || !aligned(s, 4) || !aligned(g_base, 4) || !aligned(g_meta, 4) || !aligned(p_out, 4) ||
         !aligned(sumsq_out, 8))
         return SAMA_ERR_ALIGN;
@@ -97,6 +92,18 @@ int validate_adapt(sama_ctx* ctx, int64_t n, const float* m, const float* s, con
         overlaps(p_out, bytes, g_base, bytes) || overlaps(p_out, bytes, sumsq_out, 8))
         return SAMA_ERR_OVERLAP;
     if (p_out != g_meta && overlaps(p_out, bytes, g_meta, bytes)) return SAMA_ERR_OVERLAP;
+    return SAMA_OK;
+}
+
+}  // namespace sama
+
+namespace {
+
+int check_mlp(const sama_mlp_t* mlp) {
+    if (!mlp || !mlp->dims) return SAMA_ERR_NULL;
+    if (mlp->n_layers < 1 || mlp->n_layers > kMaxLayers) return SAMA_ERR_SIZE;
+    for (int l = 0; l <= mlp->n_layers; ++l)
+        if (mlp->dims[l] < 1) return SAMA_ERR_SIZE;
     return SAMA_OK;
 }
 
@@ -274,7 +281,8 @@ int sama_destroy(sama_ctx* ctx) {
 int sama_adapt(sama_ctx* ctx, int64_t n, const float* m, const float* s, const float* g_base,
                const float* g_meta, const sama_adam_t* adam, float* p_out, double* sumsq_out, void* stream) {
     AdaptConsts c;
-    const int rc = validate_adapt(ctx, n, m, s, g_base, g_meta, adam, p_out, sumsq_out, &c);
+    if (!ctx) return SAMA_ERR_NULL;
+    const int rc = validate_adapt(ctx->max_n, n, m, s, g_base, g_meta, adam, p_out, sumsq_out, &c);
     if (rc != SAMA_OK) return rc;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return SAMA_ERR_CUDA;
@@ -320,7 +328,7 @@ int sama_step(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* thet
     if (rc != SAMA_OK) return rc;
     if (n != sama_mlp_param_count(mlp)) return SAMA_ERR_SIZE;
     AdaptConsts c;
-    rc = validate_adapt(ctx, n, m, s, g_base, g_meta, adam, p_out, nullptr, &c);
+    rc = validate_adapt(ctx->max_n, n, m, s, g_base, g_meta, adam, p_out, nullptr, &c);
     if (rc != SAMA_OK) return rc;
     rc = validate_perturb(ctx, n, theta, p_out, nullptr, alpha, theta_plus, theta_minus, nullptr);
     if (rc != SAMA_OK) return rc;

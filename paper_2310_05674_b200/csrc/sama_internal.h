@@ -86,6 +86,11 @@ struct KernelScope {
     }
 };
 
+// sama_api.cu : host-side checks of the adaptation's arguments (no launch)
+int check_adam(const sama_adam_t* a, AdaptConsts* out);
+int validate_adapt(int64_t max_n, int64_t n, const float* m, const float* s, const float* g_base,
+                   const float* g_meta, const sama_adam_t* adam, float* p_out, double* sumsq_out, AdaptConsts* c);
+
 // adapt_perturb.cu
 cudaError_t launch_adapt_sumsq(sama_ctx* ctx, int64_t n, const float* m, const float* s, const float* g_base,
                                const float* g_meta, const AdaptConsts& c, float* p_out, double* sumsq_out,
