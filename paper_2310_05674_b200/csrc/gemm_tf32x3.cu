@@ -1,0 +1,451 @@
+// Dual-branch layer of the perturbed forward pass (Eq. 5) on the 5th-generation
+// tensor cores, in arithmetic that stays faithful to fp32.
+//
+// Each fp32 operand x is carried as two TF32 numbers, hi = tf32(x) and
+// lo = tf32(x - hi), so that hi + lo holds x to about 2^-22 relative.  A product
+// A W^T is then three tensor-core products accumulated in fp32 in tensor
+// memory:  Ahi Wlo^T + Alo Whi^T + Ahi Whi^T  (the lo*lo term, 2^-22 relative, is
+// dropped).  The finite difference of Eq. 5 divides the difference of two
+// forward passes by 2 eps_fd, which amplifies rounding by 1/eps_fd; plain TF32
+// (2^-11) would drown the signal, which is why the split is needed.
+//
+// Structure of gemm_tf32x3_kernel (one 128 x BN output tile per CTA, 192 threads):
+//   warp 0    : TMA producer.  Per k-block of 32 floats it loads four tiles
+//               (A hi/lo: 128 x 32, W hi/lo: BN x 32) with cp.async.bulk.tensor
+//               into 128-byte-swizzled shared memory and signals a "full"
+//               mbarrier with the byte count.  No multicast.
+//   warp 1    : allocates tensor memory, then one lane issues, per k-block,
+//               4 k-steps x 3 tcgen05.mma kind::tf32 (M = 128, N = BN, K = 8)
+//               from shared-memory descriptors and commits to the stage's
+//               "empty" mbarrier; a last commit signals the accumulator.
+//   warps 2-5 : epilogue.  Each warp reads its 32 lanes of the accumulator with
+//               tcgen05.ld, adds the bias, applies ReLU, and either stores fp32
+//               logits or stores the next layer's hi/lo operands directly.
+// Operands are K-major in global memory ([rows][K], K padded to a multiple of
+// 32 with zeros), which is what both TMA and the K-major UMMA descriptor want.
+// Every mbarrier wait is bounded: if one expires the CTA raises
+// SAMA_DEV_TIMEOUT in the device status word, stops issuing work, waits (again
+// bounded) for the copies it has in flight, frees its tensor memory and exits.
+#include <cuda.h>
+
+#include "sama_internal.h"
+
+namespace sama {
+
+namespace {
+
+constexpr int BM = 128;       // rows of the output tile = TMEM lanes
+constexpr int BKF = 32;       // floats per k-block = one 128-byte swizzle row
+constexpr int UMMA_K = 8;     // K of one kind::tf32 instruction
+constexpr int kThreads = 192;
+constexpr long long kWaitCycles = 4000000000LL;  // ~2 s at 2 GHz
+
+__host__ __device__ constexpr int stages_for(int bn) { return bn >= 128 ? 3 : 4; }
+__host__ __device__ constexpr int stage_bytes(int bn) { return 2 * BM * BKF * 4 + 2 * bn * BKF * 4; }
+__host__ __device__ constexpr int smem_bytes(int bn) { return stages_for(bn) * stage_bytes(bn) + 1024 + 256; }
+
+// ---------------------------------------------------------------- PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within kWaitCycles.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try(bar, parity)) return true;
+        if (clock64() - t0 > kWaitCycles) return false;
+    }
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The mbarrier is signalled when every tcgen05.mma issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes
+// with the 128-byte swizzle: start address / 16 in bits [0,14), leading byte
+// offset (unused for swizzled K-major, 1) in [16,30), stride between groups of
+// 8 rows (1024 bytes) / 16 in [32,46), descriptor version 1 in [46,48), layout
+// type 2 (128-byte swizzle) in [61,64).
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+
+// Instruction descriptor: D = fp32 (1 at bit 4), A and B = TF32 (2 at bits 7 and
+// 10), both K-major (bits 15, 16 clear), N/8 at bit 17, M/16 at bit 24.
+__host__ __device__ constexpr uint32_t make_idesc(int n) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+__device__ __forceinline__ float to_tf32(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+
+struct TcArgs {
+    const float* bias[2];  // [N] fp32 (slices of theta+ / theta-), may be unaligned
+    float* out_f32[2];     // last layer: logits [M][ldc]
+    float* out_hi;         // hidden layers: next operand hi, [2][M][ld_next]
+    float* out_lo;
+    int M, N, num_kb;
+    int ldc, ld_next;      // ld_next = N rounded up to 32 (zero-filled tail)
+    int relu, last, shared_a;
+    uint32_t tx_bytes;     // bytes the four copies of one k-block deliver
+    int32_t* status;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
+                   const __grid_constant__ CUtensorMap map_w_hi, const __grid_constant__ CUtensorMap map_w_lo,
+                   TcArgs args) {
+    constexpr int STAGES = stages_for(BN);
+    constexpr int A_BYTES = BM * BKF * 4, W_BYTES = BN * BKF * 4;
+    constexpr int STAGE = stage_bytes(BN);
+    constexpr uint32_t TMEM_COLS = BN < 32 ? 32 : BN;
+    constexpr uint32_t IDESC = make_idesc(BN);
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // tiles need 1024-byte alignment
+    const uint32_t bars = base + STAGES * STAGE;                   // full[STAGES], empty[STAGES], accum, tmem slot
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+    const uint32_t accum_bar = bars + 8u * (2 * STAGES);
+    const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 1);
+    const uint32_t abort_slot = tmem_slot + 4;
+    volatile uint32_t* abort_flag =
+        reinterpret_cast<volatile uint32_t*>(smem_raw + (abort_slot - smem_u32(smem_raw)));
+    volatile uint32_t* tmem_ptr_slot =
+        reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int br = blockIdx.z;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int num_kb = args.num_kb;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        mbar_init(accum_bar, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_ptr_slot;
+
+    auto raise_timeout = [&]() {
+        *abort_flag = 1;
+        atomicOr(args.status, (int)SAMA_DEV_TIMEOUT);
+    };
+
+    if (warp == 0) {
+        // ---------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            int issued = 0;
+            const int za = args.shared_a ? 0 : br;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % STAGES;
+                const uint32_t round = kb / STAGES;
+                if (kb >= STAGES && !mbar_wait(empty_bar(s), (round - 1) & 1)) { raise_timeout(); break; }
+                if (*abort_flag) break;
+                const uint32_t st = base + s * STAGE;
+                mbar_expect_tx(full_bar(s), args.tx_bytes);
+                tma_load_3d(st, &map_a_hi, full_bar(s), kb * BKF, m0, za);
+                tma_load_3d(st + A_BYTES, &map_a_lo, full_bar(s), kb * BKF, m0, za);
+                tma_load_3d(st + 2 * A_BYTES, &map_w_hi, full_bar(s), kb * BKF, n0, br);
+                tma_load_3d(st + 2 * A_BYTES + W_BYTES, &map_w_lo, full_bar(s), kb * BKF, n0, br);
+                issued = kb + 1;
+            }
+            if (*abort_flag) {
+                // let the copies already issued land before the CTA's shared memory goes away
+                for (int kb = (issued > STAGES ? issued - STAGES : 0); kb < issued; ++kb)
+                    mbar_wait(full_bar(kb % STAGES), (kb / STAGES) & 1);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            bool ok = true;
+            for (int kb = 0; kb < num_kb && ok; ++kb) {
+                const int s = kb % STAGES;
+                if (!mbar_wait(full_bar(s), (kb / STAGES) & 1)) { raise_timeout(); ok = false; break; }
+                if (*abort_flag) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t st = base + s * STAGE;
+                const uint64_t a_hi = make_desc(st), a_lo = make_desc(st + A_BYTES);
+                const uint64_t w_hi = make_desc(st + 2 * A_BYTES), w_lo = make_desc(st + 2 * A_BYTES + W_BYTES);
+#pragma unroll
+                for (int k = 0; k < BKF / UMMA_K; ++k) {
+                    const uint64_t adv = (uint64_t)((k * UMMA_K * 4) >> 4);  // 32 bytes per k-step inside the swizzled row
+                    umma_tf32(tmem_base, a_hi + adv, w_lo + adv, IDESC, (kb | k) != 0);
+                    umma_tf32(tmem_base, a_lo + adv, w_hi + adv, IDESC, 1);
+                    umma_tf32(tmem_base, a_hi + adv, w_hi + adv, IDESC, 1);
+                }
+                umma_commit(empty_bar(s));  // frees the stage once these products have read it
+            }
+            if (ok) umma_commit(accum_bar);
+        }
+    } else {
+        // -------------------------------------------------------------- epilogue
+        const int q = warp & 3;  // a warp may only touch TMEM lanes [32 q, 32 q + 32)
+        bool ok = true;
+        if (lane == 0) {
+            // the accumulator is final when its barrier flips, or never if a producer gave up
+            const long long t0 = clock64();
+            while (!mbar_try(accum_bar, 0)) {
+                if (*abort_flag) { ok = false; break; }
+                if (clock64() - t0 > 2 * kWaitCycles) { raise_timeout(); ok = false; break; }
+            }
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (ok) {
+            tc_fence_after();
+            const int m = m0 + q * 32 + lane;
+            const float* bias = br ? args.bias[1] : args.bias[0];
+            const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+            for (int c = 0; c < BN; c += 16) {
+                float v[16];
+                tmem_ld16(lane_addr + c, v);   // all lanes take part (sync.aligned)
+                const int n = n0 + c;
+                if (m < args.M) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        float x = v[j] + ((n + j < args.N) ? bias[n + j] : 0.f);
+                        if (args.relu && x < 0.f) x = 0.f;
+                        v[j] = x;
+                    }
+                    if (args.last) {
+                        float* dst = (br ? args.out_f32[1] : args.out_f32[0]) + (int64_t)m * args.ldc + n;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (n + j < args.N) dst[j] = v[j];
+                    } else if (n < args.ld_next) {
+                        // columns in [N, ld_next) are the next layer's zero padding along K
+                        const int64_t off = ((int64_t)br * args.M + m) * args.ld_next + n;
+                        float hi[16], lo[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const float x = (n + j < args.N) ? v[j] : 0.f;
+                            hi[j] = to_tf32(x);
+                            lo[j] = to_tf32(x - hi[j]);
+                        }
+                        float4* dh = reinterpret_cast<float4*>(args.out_hi + off);
+                        float4* dl = reinterpret_cast<float4*>(args.out_lo + off);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            dh[j] = make_float4(hi[4 * j], hi[4 * j + 1], hi[4 * j + 2], hi[4 * j + 3]);
+                            dl[j] = make_float4(lo[4 * j], lo[4 * j + 1], lo[4 * j + 2], lo[4 * j + 3]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// Splits rows of an fp32 matrix into TF32 hi / lo with the row length padded to
+// ld_out (zeros).  grid.z selects the branch (source pointer and output slab).
+struct SplitArgs {
+    const float* src[2];
+    int64_t rows, cols;
+    int ld_src, ld_out;
+    float* hi;
+    float* lo;
+};
+
+__global__ void __launch_bounds__(256)
+split_tf32_kernel(SplitArgs a) {
+    const int br = blockIdx.z;
+    const float* __restrict__ src = br ? a.src[1] : a.src[0];
+    const int64_t total = a.rows * a.ld_out;
+    float* __restrict__ hi = a.hi + (int64_t)br * total;
+    float* __restrict__ lo = a.lo + (int64_t)br * total;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int64_t r = i / a.ld_out;
+        const int c = (int)(i - r * a.ld_out);
+        const float x = c < a.cols ? src[r * a.ld_src + c] : 0.f;
+        const float h = to_tf32(x);
+        hi[i] = h;
+        lo[i] = to_tf32(x - h);
+    }
+}
+
+// ------------------------------------------------------------------ host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// 3-D map over [slabs][rows][ld] fp32 with a box of 32 floats x box_rows rows, 128-byte swizzle, zero fill.
+bool make_map(CUtensorMap* map, const float* base, int ld, int64_t rows, int slabs, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)ld, (cuuint64_t)rows, (cuuint64_t)slabs};
+    cuuint64_t strides[2] = {(cuuint64_t)ld * 4, (cuuint64_t)ld * 4 * (cuuint64_t)rows};
+    cuuint32_t box[3] = {(cuuint32_t)BKF, (cuuint32_t)box_rows, 1};  // caller keeps box_rows <= rows
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN>
+cudaError_t launch_tc(const CUtensorMap maps[4], const TcArgs& a, dim3 grid, cudaStream_t st) {
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_tf32x3_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             smem_bytes(BN));
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    gemm_tf32x3_kernel<BN><<<grid, kThreads, smem_bytes(BN), st>>>(maps[0], maps[1], maps[2], maps[3], a);
+    return cudaGetLastError();
+}
+
+inline int round_up32(int x) { return (x + 31) & ~31; }
+
+}  // namespace
+
+cudaError_t launch_split_tf32(sama_ctx* ctx, const float* src0, const float* src1, int branches, int64_t rows,
+                              int cols, int ld_src, float* hi, float* lo, cudaStream_t st) {
+    SplitArgs a;
+    a.src[0] = src0;
+    a.src[1] = src1;
+    a.rows = rows;
+    a.cols = cols;
+    a.ld_src = ld_src;
+    a.ld_out = round_up32(cols);
+    a.hi = hi;
+    a.lo = lo;
+    const int64_t total = rows * a.ld_out;
+    int64_t blocks = (total + 256 * 4 - 1) / (256 * 4);
+    const int64_t cap = (int64_t)ctx->sm_count * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    KernelScope scope(ctx, SAMA_K_SPLIT, -1, st);
+    split_tf32_kernel<<<dim3((unsigned)blocks, 1, branches), 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+// One layer on the tensor cores.  a_hi/a_lo: [shared_a ? 1 : 2][M][Kp]; w_hi/w_lo: [2][N][Kp]; Kp = K rounded
+// up to 32.  Hidden layers write the next operands (out_hi/out_lo, [2][M][round_up32(N)]); the last layer
+// writes fp32 logits.
+cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st) {
+    const int Kp = round_up32(L.K);
+    // N-tile: 16 for a narrow last layer; 64 when 128-wide tiles would leave SMs idle; else 128.
+    // (Hidden layers never take 16: their tiles must also write the zero padding up to round_up32(N).)
+    const int64_t tiles128 = (int64_t)((L.M + BM - 1) / BM) * ((L.N + 127) / 128) * 2;
+    const int bn = (L.last && L.N <= 16) ? 16 : ((L.N <= 64 || tiles128 < ctx->sm_count) ? 64 : 128);
+    CUtensorMap maps[4];
+    const int a_slabs = L.shared_a ? 1 : 2;
+    // a box never exceeds the tensor's extent; rows of the shared-memory tile that no copy fills only
+    // feed output rows / columns that the epilogue does not store
+    const int a_box = L.M < BM ? L.M : BM, w_box = L.N < bn ? L.N : bn;
+    if (!make_map(&maps[0], L.a_hi, Kp, L.M, a_slabs, a_box) || !make_map(&maps[1], L.a_lo, Kp, L.M, a_slabs, a_box) ||
+        !make_map(&maps[2], L.w_hi, Kp, L.N, 2, w_box) || !make_map(&maps[3], L.w_lo, Kp, L.N, 2, w_box))
+        return cudaErrorInvalidValue;
+    TcArgs a;
+    a.bias[0] = L.bias[0];
+    a.bias[1] = L.bias[1];
+    a.out_f32[0] = L.out_f32[0];
+    a.out_f32[1] = L.out_f32[1];
+    a.out_hi = L.out_hi;
+    a.out_lo = L.out_lo;
+    a.M = L.M;
+    a.N = L.N;
+    a.num_kb = Kp / BKF;
+    a.ldc = L.ldc;
+    a.ld_next = round_up32(L.N);
+    a.relu = L.relu;
+    a.last = L.last;
+    a.shared_a = L.shared_a;
+    a.tx_bytes = (uint32_t)(2 * a_box * BKF * 4 + 2 * w_box * BKF * 4);
+    a.status = &ctx->scalars->status;
+    dim3 grid((L.N + bn - 1) / bn, (L.M + BM - 1) / BM, 2);
+    KernelScope scope(ctx, SAMA_K_GEMM_TF32X3, L.layer, st);
+    if (bn == 16) return launch_tc<16>(maps, a, grid, st);
+    if (bn == 64) return launch_tc<64>(maps, a, grid, st);
+    return launch_tc<128>(maps, a, grid, st);
+}
+
+}  // namespace sama

@@ -154,11 +154,77 @@ int validate_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, c
     return SAMA_OK;
 }
 
+// Whether this model fits the operand-split workspace of the tensor-core path.
+bool tc_fits(const sama_ctx* ctx, const sama_mlp_t* mlp, int32_t B) {
+    auto r32 = [](int x) { return (size_t)((x + 31) & ~31); };
+    const int L = mlp->n_layers;
+    if (ctx->x_split_half == 0 || (size_t)B * r32(mlp->dims[0]) > ctx->x_split_half) return false;
+    for (int l = 0; l < L; ++l) {
+        if (2 * (size_t)mlp->dims[l + 1] * r32(mlp->dims[l]) > ctx->w_split_half) return false;
+        if (l + 1 < L && 2 * (size_t)B * r32(mlp->dims[l + 1]) > ctx->a_split_half) return false;
+    }
+    return true;
+}
+
+// Forward pass of both branches on the tensor cores (3xTF32): operands are split into TF32 hi/lo
+// (X once, each layer's W+- before its product; hidden activations are split by the producing epilogue).
+int run_forward_tc(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const float* theta_minus,
+                   const float* X, int32_t B, cudaStream_t st) {
+    const int L = mlp->n_layers;
+    SAMA_CUDA(ctx, launch_split_tf32(ctx, X, X, 1, B, mlp->dims[0], mlp->dims[0], ctx->x_split,
+                                     ctx->x_split + ctx->x_split_half, st));
+    int64_t off = 0;
+    for (int l = 0; l < L; ++l) {
+        const int din = mlp->dims[l], dout = mlp->dims[l + 1];
+        const bool last = (l + 1 == L);
+        SAMA_CUDA(ctx, launch_split_tf32(ctx, theta_plus + off, theta_minus + off, 2, dout, din, din, ctx->w_split,
+                                         ctx->w_split + ctx->w_split_half, st));
+        TcLayer t;
+        if (l == 0) {
+            t.a_hi = ctx->x_split;
+            t.a_lo = ctx->x_split + ctx->x_split_half;
+        } else {
+            t.a_hi = ctx->a_split[(l - 1) & 1];
+            t.a_lo = ctx->a_split[(l - 1) & 1] + ctx->a_split_half;
+        }
+        t.w_hi = ctx->w_split;
+        t.w_lo = ctx->w_split + ctx->w_split_half;
+        t.bias[0] = theta_plus + off + (int64_t)din * dout;
+        t.bias[1] = theta_minus + off + (int64_t)din * dout;
+        t.out_f32[0] = ctx->logits;
+        t.out_f32[1] = ctx->logits + (int64_t)B * dout;
+        t.out_hi = last ? nullptr : ctx->a_split[l & 1];
+        t.out_lo = last ? nullptr : ctx->a_split[l & 1] + ctx->a_split_half;
+        t.M = B;
+        t.N = dout;
+        t.K = din;
+        t.ldc = dout;
+        t.relu = last ? 0 : 1;
+        t.last = last ? 1 : 0;
+        t.shared_a = (l == 0) ? 1 : 0;
+        t.layer = l;
+        SAMA_CUDA(ctx, launch_gemm_tf32x3(ctx, t, st));
+        off += (int64_t)din * dout + dout;
+    }
+    return SAMA_OK;
+}
+
 // The dual-branch forward and the finite difference, arguments already validated.
 int run_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const float* theta_minus,
            const float* X, const int32_t* y, const float* lambda, int32_t B, const float* eps_fd,
            float* metagrad_out, float* loss_plus_out, float* loss_minus_out, cudaStream_t st) {
     const int L = mlp->n_layers;
+    const int C = mlp->dims[L];
+    const bool fits = tc_fits(ctx, mlp, B);
+    if (ctx->gemm_mode == 2 && !fits) return SAMA_ERR_SIZE;
+    if (ctx->gemm_mode != 1 && fits) {
+        const int rc = run_forward_tc(ctx, mlp, theta_plus, theta_minus, X, B, st);
+        if (rc != SAMA_OK) return rc;
+        SAMA_CUDA(ctx, launch_ce_fd(ctx, ctx->logits, ctx->logits + (int64_t)B * C, C, y, lambda, B, C,
+                                    eps_fd ? eps_fd : &ctx->scalars->eps_fd, metagrad_out, loss_plus_out,
+                                    loss_minus_out, st));
+        return SAMA_OK;
+    }
     const float* in[2] = {X, X};
     int ld_in = mlp->dims[0];
     int64_t off = 0;
@@ -189,7 +255,6 @@ int run_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const 
         ld_in = dout;
         off += (int64_t)din * dout + dout;
     }
-    const int C = mlp->dims[L];
     SAMA_CUDA(ctx, launch_ce_fd(ctx, in[0], in[1], C, y, lambda, B, C, eps_fd ? eps_fd : &ctx->scalars->eps_fd,
                                 metagrad_out, loss_plus_out, loss_minus_out, st));
     return SAMA_OK;
@@ -251,6 +316,22 @@ int sama_create(sama_ctx** out, int device, int64_t max_n, int32_t max_batch, co
             ok = cudaMalloc(&ctx->act[0], bytes) == cudaSuccess && cudaMalloc(&ctx->act[1], bytes) == cudaSuccess;
         }
         ok = ok && cudaMalloc(&ctx->logits, sizeof(float) * 2 * (size_t)max_batch * ctx->max_classes) == cudaSuccess;
+        // operand splits of the tensor-core path
+        auto r32 = [](int x) { return (size_t)((x + 31) & ~31); };
+        size_t wmax = 0, amax = 0;
+        for (int l = 0; l < L; ++l) {
+            const size_t we = (size_t)mlp->dims[l + 1] * r32(mlp->dims[l]);
+            wmax = we > wmax ? we : wmax;
+            if (l + 1 < L) { const size_t ae = r32(mlp->dims[l + 1]); amax = ae > amax ? ae : amax; }
+        }
+        ctx->x_split_half = (size_t)max_batch * r32(mlp->dims[0]);
+        ctx->w_split_half = 2 * wmax;
+        ctx->a_split_half = 2 * (size_t)max_batch * amax;
+        ok = ok && cudaMalloc(&ctx->x_split, sizeof(float) * 2 * ctx->x_split_half) == cudaSuccess &&
+             cudaMalloc(&ctx->w_split, sizeof(float) * 2 * ctx->w_split_half) == cudaSuccess;
+        if (ok && amax > 0)
+            ok = cudaMalloc(&ctx->a_split[0], sizeof(float) * 2 * ctx->a_split_half) == cudaSuccess &&
+                 cudaMalloc(&ctx->a_split[1], sizeof(float) * 2 * ctx->a_split_half) == cudaSuccess;
     }
     if (!ok || cudaDeviceSynchronize() != cudaSuccess) {
         cudaGetLastError();
@@ -269,6 +350,10 @@ int sama_destroy(sama_ctx* ctx) {
     cudaFree(ctx->act[0]);
     cudaFree(ctx->act[1]);
     cudaFree(ctx->logits);
+    cudaFree(ctx->x_split);
+    cudaFree(ctx->w_split);
+    cudaFree(ctx->a_split[0]);
+    cudaFree(ctx->a_split[1]);
     cudaFree(ctx->stage);
     if (ctx->prof) {
         for (auto& r : ctx->prof->records) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
@@ -444,7 +529,6 @@ int sama_last_cuda_error(sama_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0;
 int sama_set_gemm_mode(sama_ctx* ctx, int mode) {
     if (!ctx) return SAMA_ERR_NULL;
     if (mode < 0 || mode > 2) return SAMA_ERR_PARAM;
-    if (mode == 2) return SAMA_ERR_UNSUPPORTED;
     ctx->gemm_mode = mode;
     return SAMA_OK;
 }

@@ -58,6 +58,11 @@ struct sama_ctx {
     double* partials;              // device [kMaxPartials]
     float* act[2];                 // device: ping-pong activations, each [2][max_batch][max_width]
     float* logits;                 // device [2][max_batch][max_classes]
+    // TF32 hi/lo operand splits of the tensor-core path, each buffer holds hi then lo
+    float* x_split;                // device [2][max_batch][round32(d_0)]
+    float* w_split;                // device [2][2][max_l d_l round32(d_{l-1})]
+    float* a_split[2];             // device, ping-pong: [2][2][max_batch][round32(max hidden)]
+    size_t x_split_half, w_split_half, a_split_half;  // floats per hi (or lo) part; 0 = path unavailable
     float* stage;                  // device: staging of the host entry point (allocated on first use)
     size_t stage_bytes;
     sama::Profiler* prof;          // host
@@ -114,6 +119,23 @@ struct GemmArgs {
 cudaError_t launch_gemm_ffma(sama_ctx* ctx, const GemmArgs& g, cudaStream_t st);
 // sama_api.cu : picks the matrix-product path of one layer
 cudaError_t launch_gemm(sama_ctx* ctx, const GemmArgs& g, cudaStream_t st);
+
+// gemm_tf32x3.cu : tensor-core path (3xTF32)
+struct TcLayer {
+    const float* a_hi;     // [shared_a ? 1 : 2][M][round32(K)]
+    const float* a_lo;
+    const float* w_hi;     // [2][N][round32(K)]
+    const float* w_lo;
+    const float* bias[2];  // [N]
+    float* out_f32[2];     // last layer: [M][ldc]
+    float* out_hi;         // hidden layers: [2][M][round32(N)]
+    float* out_lo;
+    int M, N, K, ldc;
+    int relu, last, shared_a, layer;
+};
+cudaError_t launch_split_tf32(sama_ctx* ctx, const float* src0, const float* src1, int branches, int64_t rows,
+                              int cols, int ld_src, float* hi, float* lo, cudaStream_t st);
+cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st);
 
 // ce_fd.cu
 cudaError_t launch_ce_fd(sama_ctx* ctx, const float* z_plus, const float* z_minus, int ldz, const int32_t* y,

@@ -30,9 +30,11 @@ def unaligned(a: np.ndarray, shift: int = 1) -> torch.Tensor:
 
 
 class Ctx:
-    def __init__(self, max_n, max_batch=0, dims=None):
+    def __init__(self, max_n, max_batch=0, dims=None, gemm_mode=0):
         self.mlp = B.MLP(dims) if dims is not None else None
         self.h = B.sama_create(0, max_n, max_batch, self.mlp)
+        if gemm_mode:
+            B.sama_set_gemm_mode(self.h, gemm_mode)
 
     def close(self):
         if self.h:

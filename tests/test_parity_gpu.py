@@ -138,11 +138,16 @@ def test_perturb_degenerate_norm_sets_status():
 
 # ---------------------------------------------------- forward + FD alone ----
 
-RAGGED = [((12, 5), 1), ((33, 17, 12, 6), 7), ((100, 50, 3), 129), ((257, 130, 66, 11), 65), ((64, 64, 64, 16), 300)]
+RAGGED = [((12, 5), 1), ((33, 17, 12, 6), 7), ((100, 50, 3), 129), ((257, 130, 66, 11), 65), ((64, 64, 64, 16), 300),
+          ((40, 200, 72, 24), 257)]
+
+# 1 = fp32 FMA on the CUDA cores, 2 = tensor cores (three TF32 products per fp32 product)
+GEMM_MODES = [1, 2]
 
 
+@pytest.mark.parametrize("gemm_mode", GEMM_MODES)
 @pytest.mark.parametrize("dims,batch", RAGGED)
-def test_fd_metagrad_parity_ragged(dims, batch):
+def test_fd_metagrad_parity_ragged(dims, batch, gemm_mode):
     cfg, w = W.custom_mlp(dims, batch, seed=sum(dims))
     n = cfg.n_params
     # non-zero biases and a realistic pair theta+-
@@ -153,7 +158,7 @@ def test_fd_metagrad_parity_ragged(dims, batch):
     lp = oracle.losses(dims, tp_np, w["X"], w["y"])
     lm = oracle.losses(dims, tm_np, w["X"], w["y"])
     ref = oracle.fd(lp, lm, w["lam"], float(eps_val), batch)
-    with Ctx(n, batch, dims) as ctx:
+    with Ctx(n, batch, dims, gemm_mode) as ctx:
         out = [torch.empty(batch, dtype=torch.float32, device=DEV) for _ in range(3)]
         B.sama_fd_metagrad(ctx.h, ctx.mlp, dev(tp_np), dev(tm_np), dev(w["X"]), dev(w["y"]), dev(w["lam"]), batch,
                            dev(np.array([eps_val])), out[0], out[1], out[2])
@@ -187,13 +192,21 @@ def test_bad_label_is_reported_not_faulted():
 
 # ------------------------------------------------------------ whole step ----
 
-def check_step(cfg, w, adam, alpha, rows=None, use_gbase=True):
-    """Runs sama_step on the full batch; the checker runs on ``rows`` (all if None)."""
-    with Ctx(cfg.n_params, cfg.batch, cfg.dims) as ctx:
+_REF_CACHE = {}
+
+
+def check_step(cfg, w, adam, alpha, rows=None, use_gbase=True, gemm_mode=0, key=None):
+    """Runs sama_step on the full batch; the checker runs on ``rows`` (all if None).
+    ``key`` caches the checker's result across the gemm modes of one workload."""
+    with Ctx(cfg.n_params, cfg.batch, cfg.dims, gemm_mode) as ctx:
         got = run_step(ctx, cfg, w, adam, alpha, use_gbase=use_gbase)
     sel = slice(None) if rows is None else rows
-    ref = oracle.step(cfg.dims, w["theta"], w["m"], w["s"], w["g_base"] if use_gbase else None, w["g_meta"],
-                      o_adam(adam), alpha, w["X"][sel], w["y"][sel], w["lam"][sel], B_norm=cfg.batch)
+    ref = _REF_CACHE.get(key) if key else None
+    if ref is None:
+        ref = oracle.step(cfg.dims, w["theta"], w["m"], w["s"], w["g_base"] if use_gbase else None, w["g_meta"],
+                          o_adam(adam), alpha, w["X"][sel], w["y"][sel], w["lam"][sel], B_norm=cfg.batch)
+        if key:
+            _REF_CACHE[key] = ref
     assert got["status"] == 0 and not ref["degenerate"]
     assert_adapt_close(got["p"], ref["p"])
     assert got["eps_fd"] == pytest.approx(ref["eps_fd"], rel=1e-6)
@@ -205,53 +218,59 @@ def check_step(cfg, w, adam, alpha, rows=None, use_gbase=True):
     dq = (got["loss_plus"].astype(np.float64) - got["loss_minus"].astype(np.float64))[sel]
     dr = ref["loss_plus"] - ref["loss_minus"]
     e["dq_norm_rel"] = float(np.linalg.norm(dq - dr) / np.linalg.norm(dr))
-    print("\n[parity] %s alpha=%g: %s" % (cfg.name, alpha, e))
+    print("\n[parity] %s alpha=%g gemm_mode=%d: %s" % (cfg.name, alpha, gemm_mode, e))
     return e
 
 
+@pytest.mark.parametrize("gemm_mode", GEMM_MODES)
 @pytest.mark.parametrize("alpha", [1e-2, 1.0])
-def test_step_parity_tiny(alpha):
+def test_step_parity_tiny(alpha, gemm_mode):
     cfg = W.CONFIGS["tiny"]
-    check_step(cfg, W.mlp_workload(cfg, 0), B.Adam(), alpha)
+    check_step(cfg, W.mlp_workload(cfg, 0), B.Adam(), alpha, gemm_mode=gemm_mode, key=("tiny", alpha))
 
 
-def test_step_parity_tiny_variants():
+@pytest.mark.parametrize("gemm_mode", GEMM_MODES)
+def test_step_parity_tiny_variants(gemm_mode):
     cfg = W.CONFIGS["tiny"]
     w = W.mlp_workload(cfg, 0)
-    check_step(cfg, w, B.Adam(), 1e-2, use_gbase=False)
-    check_step(cfg, w, B.Adam(identity=True), 1.0)
-    check_step(cfg, w, B.Adam(step=1, drop_eps_term=True), 1e-2)
-    check_step(cfg, w, B.Adam(bias_correction=False), 1.0, use_gbase=False)
+    check_step(cfg, w, B.Adam(), 1e-2, use_gbase=False, gemm_mode=gemm_mode, key=("tiny", "nog"))
+    check_step(cfg, w, B.Adam(identity=True), 1.0, gemm_mode=gemm_mode, key=("tiny", "id"))
+    check_step(cfg, w, B.Adam(step=1, drop_eps_term=True), 1e-2, gemm_mode=gemm_mode, key=("tiny", "drop"))
+    check_step(cfg, w, B.Adam(bias_correction=False), 1.0, use_gbase=False, gemm_mode=gemm_mode, key=("tiny", "nobias"))
 
 
+@pytest.mark.parametrize("gemm_mode", GEMM_MODES)
 @pytest.mark.parametrize("dims,batch", RAGGED[1:])
-def test_step_parity_ragged(dims, batch):
+def test_step_parity_ragged(dims, batch, gemm_mode):
     cfg, w = W.custom_mlp(dims, batch, seed=3 + sum(dims))
-    check_step(cfg, w, B.Adam(), 1e-2)
+    check_step(cfg, w, B.Adam(), 1e-2, gemm_mode=gemm_mode, key=("ragged", dims, batch))
 
 
-def test_step_parity_mlp3072():
+@pytest.mark.parametrize("gemm_mode", GEMM_MODES)
+def test_step_parity_mlp3072(gemm_mode):
     cfg = W.CONFIGS["mlp3072"]
     w = W.mlp_workload(cfg, 0)
-    check_step(cfg, w, B.Adam(), 1e-2)
-    check_step(cfg, w, B.Adam(), 1.0, rows=np.arange(0, cfg.batch, 8))
+    check_step(cfg, w, B.Adam(), 1e-2, gemm_mode=gemm_mode, key=("mlp3072", 1e-2))
+    check_step(cfg, w, B.Adam(), 1.0, rows=np.arange(0, cfg.batch, 8), gemm_mode=gemm_mode, key=("mlp3072", 1.0))
 
 
-def test_step_parity_head1024():
+@pytest.mark.parametrize("gemm_mode", GEMM_MODES)
+def test_step_parity_head1024(gemm_mode):
     cfg = W.CONFIGS["head1024"]
     w = W.mlp_workload(cfg, 0)
-    check_step(cfg, w, B.Adam(), 1e-2)
-    check_step(cfg, w, B.Adam(), 1.0, rows=np.arange(0, cfg.batch, 64))
+    check_step(cfg, w, B.Adam(), 1e-2, gemm_mode=gemm_mode, key=("head1024", 1e-2))
+    check_step(cfg, w, B.Adam(), 1.0, rows=np.arange(0, cfg.batch, 64), gemm_mode=gemm_mode, key=("head1024", 1.0))
 
 
-def test_step_parity_wide4096_sampled():
+@pytest.mark.parametrize("gemm_mode", GEMM_MODES)
+def test_step_parity_wide4096_sampled(gemm_mode):
     """Full-size launch; the checker evaluates a sample of the rows (each output
     depends only on its own row given theta+-, which are compared in full)."""
     cfg = W.CONFIGS["wide4096"]
     w = W.mlp_workload(cfg, 0)
     rows = np.unique(np.concatenate([np.arange(0, cfg.batch, 97), [cfg.batch - 1]]))
-    check_step(cfg, w, B.Adam(), 1e-2, rows=rows)
-    check_step(cfg, w, B.Adam(), 1.0, rows=rows[::2])
+    check_step(cfg, w, B.Adam(), 1e-2, rows=rows, gemm_mode=gemm_mode, key=("wide4096", 1e-2))
+    check_step(cfg, w, B.Adam(), 1.0, rows=rows[::2], gemm_mode=gemm_mode, key=("wide4096", 1.0))
 
 
 def test_step_host_matches_step():
