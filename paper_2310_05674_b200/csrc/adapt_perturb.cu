@@ -270,6 +270,93 @@ perturb_kernel(int64_t n, const float* theta, const float* __restrict__ p, const
     }
 }
 
+__device__ __forceinline__ float tf32_round(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+__device__ __forceinline__ void tf32_split(float4 x, float4& h, float4& l) {
+    h.x = tf32_round(x.x); l.x = tf32_round(x.x - h.x);
+    h.y = tf32_round(x.y); l.y = tf32_round(x.y - h.y);
+    h.z = tf32_round(x.z); l.z = tf32_round(x.z - h.z);
+    h.w = tf32_round(x.w); l.w = tf32_round(x.w - h.w);
+}
+
+// perturb (Sec. 3.2) fused with the operand preparation of the tensor-core
+// forward pass: besides theta+ and theta-, every weight element is written as
+// TF32 hi / lo into the row-padded split buffers of both branches, so the
+// forward pass needs no further sweep over the parameters.  32 B/element.
+// Preconditions (checked on the host): 16-byte aligned pointers, every weight
+// block starts at a multiple of 4 and has K % 4 == 0 and fewer than 2^31 elements.
+__global__ void __launch_bounds__(kThreads)
+perturb_split_kernel(int64_t n, const float* theta, const float* __restrict__ p, const double* __restrict__ sumsq,
+                     float alpha, float* theta_plus, float* theta_minus, DeviceScalars* sc, float* eps_fd_out,
+                     SplitLayout lay, float* __restrict__ hi, float* __restrict__ lo) {
+    bool bad;
+    const float eps = step_size(*sumsq, alpha, bad);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        sc->eps_fd = eps;
+        if (eps_fd_out) *eps_fd_out = eps;
+        if (bad) atomicOr(&sc->status, (int)SAMA_DEV_DEGENERATE_NORM);
+    }
+    const int64_t stride = (int64_t)gridDim.x * kThreads;
+    const int64_t items = n >> 2;
+    const float4* t4 = reinterpret_cast<const float4*>(theta);
+    const float4* p4 = reinterpret_cast<const float4*>(p);
+    float4* tp4 = reinterpret_cast<float4*>(theta_plus);
+    float4* tm4 = reinterpret_cast<float4*>(theta_minus);
+
+    auto emit = [&](int64_t i, float4 vt, float4 vp) {
+        float4 a, b;
+        plus_minus(eps, vt, vp, a, b);
+        tp4[i] = a;
+        tm4[i] = b;
+        const int64_t e = i << 2;
+        int l = -1;
+#pragma unroll 1
+        for (int k = 0; k < lay.n_layers; ++k)
+            if (e >= lay.w_off[k] && e < lay.w_off[k] + lay.w_cnt[k]) { l = k; break; }
+        if (l < 0) return;  // a bias
+        const uint32_t rel = (uint32_t)(e - lay.w_off[l]);
+        const uint32_t K = (uint32_t)lay.K[l], Kp = (uint32_t)lay.Kp[l];
+        const uint32_t row = rel / K, col = rel - row * K;
+        const int64_t dst = lay.s_off[l] + (int64_t)row * Kp + col;
+        float4 h, q;
+        tf32_split(a, h, q);
+        *reinterpret_cast<float4*>(hi + dst) = h;
+        *reinterpret_cast<float4*>(lo + dst) = q;
+        tf32_split(b, h, q);
+        *reinterpret_cast<float4*>(hi + lay.slab + dst) = h;
+        *reinterpret_cast<float4*>(lo + lay.slab + dst) = q;
+        if (Kp != K && col + 4 == K) {  // this thread closes the row: zero its padding
+            const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (uint32_t c = 4; c < Kp - K + 4; c += 4) {
+                *reinterpret_cast<float4*>(hi + dst + c) = z;
+                *reinterpret_cast<float4*>(lo + dst + c) = z;
+                *reinterpret_cast<float4*>(hi + lay.slab + dst + c) = z;
+                *reinterpret_cast<float4*>(lo + lay.slab + dst + c) = z;
+            }
+        }
+    };
+
+    int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    for (; i + stride < items; i += stride * 2) {
+        const float4 vt0 = ld_stream(t4 + i), vp0 = ld_stream(p4 + i);
+        const float4 vt1 = ld_stream(t4 + i + stride), vp1 = ld_stream(p4 + i + stride);
+        emit(i, vt0, vp0);
+        emit(i + stride, vt1, vp1);
+    }
+    for (; i < items; i += stride) emit(i, ld_stream(t4 + i), ld_stream(p4 + i));
+    if (blockIdx.x == 0) {  // n % 4 trailing elements: never weights under the preconditions
+        const int64_t k = (items << 2) + threadIdx.x;
+        if (k < n) {
+            const float t = theta[k], q = p[k];
+            theta_plus[k] = eps == 0.0f ? t : fmaf(eps, q, t);
+            theta_minus[k] = eps == 0.0f ? t : fmaf(-eps, q, t);
+        }
+    }
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 inline int stream_grid(const sama_ctx* ctx, int64_t work_items, int per_thread) {
@@ -329,6 +416,23 @@ cudaError_t launch_perturb(sama_ctx* ctx, int64_t n, const float* theta, const f
     else
         perturb_kernel<false><<<stream_grid(ctx, n, 4), kThreads, 0, st>>>(
             n, theta, p, sumsq, alpha, theta_plus, theta_minus, ctx->scalars, eps_fd_out);
+    return cudaGetLastError();
+}
+
+bool perturb_split_applicable(const SplitLayout& lay, const float* theta, const float* p, const float* theta_plus,
+                              const float* theta_minus) {
+    if (!aligned16(theta) || !aligned16(p) || !aligned16(theta_plus) || !aligned16(theta_minus)) return false;
+    for (int l = 0; l < lay.n_layers; ++l)
+        if ((lay.w_off[l] & 3) || (lay.K[l] & 3) || lay.w_cnt[l] >= ((int64_t)1 << 31)) return false;
+    return true;
+}
+
+cudaError_t launch_perturb_split(sama_ctx* ctx, int64_t n, const float* theta, const float* p, const double* sumsq,
+                                 float alpha, float* theta_plus, float* theta_minus, float* eps_fd_out,
+                                 const SplitLayout& lay, float* hi, float* lo, cudaStream_t st) {
+    KernelScope scope(ctx, SAMA_K_PERTURB, -1, st);
+    perturb_split_kernel<<<stream_grid(ctx, n >> 2, kUnroll), kThreads, 0, st>>>(
+        n, theta, p, sumsq, alpha, theta_plus, theta_minus, ctx->scalars, eps_fd_out, lay, hi, lo);
     return cudaGetLastError();
 }
 

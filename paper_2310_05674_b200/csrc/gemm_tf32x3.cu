@@ -310,31 +310,52 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     }
 }
 
-// Splits rows of an fp32 matrix into TF32 hi / lo with the row length padded to
-// ld_out (zeros).  grid.z selects the branch (source pointer and output slab).
+// Splits rows of a dense fp32 matrix [rows][cols] into TF32 hi / lo with the row
+// length padded to ld_out (zeros).  grid.z selects the branch (source pointer
+// and output slab).
 struct SplitArgs {
     const float* src[2];
-    int64_t rows, cols;
-    int ld_src, ld_out;
+    int64_t rows, cols, slab;
+    int ld_out;
     float* hi;
     float* lo;
 };
 
+template <bool VEC>
 __global__ void __launch_bounds__(256)
 split_tf32_kernel(SplitArgs a) {
     const int br = blockIdx.z;
     const float* __restrict__ src = br ? a.src[1] : a.src[0];
-    const int64_t total = a.rows * a.ld_out;
-    float* __restrict__ hi = a.hi + (int64_t)br * total;
-    float* __restrict__ lo = a.lo + (int64_t)br * total;
+    float* __restrict__ hi = a.hi + (int64_t)br * a.slab;
+    float* __restrict__ lo = a.lo + (int64_t)br * a.slab;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
-        const int64_t r = i / a.ld_out;
-        const int c = (int)(i - r * a.ld_out);
-        const float x = c < a.cols ? src[r * a.ld_src + c] : 0.f;
-        const float h = to_tf32(x);
-        hi[i] = h;
-        lo[i] = to_tf32(x - h);
+    if (VEC) {
+        // cols % 4 == 0 and src 16-byte aligned: one float4 of a row per thread
+        const int q = a.ld_out >> 2;
+        const int64_t total = a.rows * q;
+        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+            const int64_t r = i / q;
+            const int c = (int)(i - r * q) << 2;
+            float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c < a.cols) x = __ldg(reinterpret_cast<const float4*>(src + r * a.cols + c));
+            float4 h, l;
+            h.x = to_tf32(x.x); l.x = to_tf32(x.x - h.x);
+            h.y = to_tf32(x.y); l.y = to_tf32(x.y - h.y);
+            h.z = to_tf32(x.z); l.z = to_tf32(x.z - h.z);
+            h.w = to_tf32(x.w); l.w = to_tf32(x.w - h.w);
+            *reinterpret_cast<float4*>(hi + r * a.ld_out + c) = h;
+            *reinterpret_cast<float4*>(lo + r * a.ld_out + c) = l;
+        }
+    } else {
+        const int64_t total = a.rows * a.ld_out;
+        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+            const int64_t r = i / a.ld_out;
+            const int c = (int)(i - r * a.ld_out);
+            const float x = c < a.cols ? src[r * a.cols + c] : 0.f;
+            const float h = to_tf32(x);
+            hi[i] = h;
+            lo[i] = to_tf32(x - h);
+        }
     }
 }
 
@@ -357,11 +378,11 @@ EncodeTiledFn encode_fn() {
 }
 
 // 3-D map over [slabs][rows][ld] fp32 with a box of 32 floats x box_rows rows, 128-byte swizzle, zero fill.
-bool make_map(CUtensorMap* map, const float* base, int ld, int64_t rows, int slabs, int box_rows) {
+bool make_map(CUtensorMap* map, const float* base, int ld, int64_t rows, int slabs, int box_rows, int64_t slab) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[3] = {(cuuint64_t)ld, (cuuint64_t)rows, (cuuint64_t)slabs};
-    cuuint64_t strides[2] = {(cuuint64_t)ld * 4, (cuuint64_t)ld * 4 * (cuuint64_t)rows};
+    cuuint64_t strides[2] = {(cuuint64_t)ld * 4, (cuuint64_t)slab * 4};
     cuuint32_t box[3] = {(cuuint32_t)BKF, (cuuint32_t)box_rows, 1};  // caller keeps box_rows <= rows
     cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, estr,
@@ -387,23 +408,28 @@ inline int round_up32(int x) { return (x + 31) & ~31; }
 }  // namespace
 
 cudaError_t launch_split_tf32(sama_ctx* ctx, const float* src0, const float* src1, int branches, int64_t rows,
-                              int cols, int ld_src, float* hi, float* lo, cudaStream_t st) {
+                              int cols, float* hi, float* lo, int64_t slab, cudaStream_t st) {
     SplitArgs a;
     a.src[0] = src0;
     a.src[1] = src1;
     a.rows = rows;
     a.cols = cols;
-    a.ld_src = ld_src;
+    a.slab = slab;
     a.ld_out = round_up32(cols);
     a.hi = hi;
     a.lo = lo;
-    const int64_t total = rows * a.ld_out;
-    int64_t blocks = (total + 256 * 4 - 1) / (256 * 4);
+    const bool vec = (cols % 4 == 0) && ((reinterpret_cast<uintptr_t>(src0) & 15u) == 0) &&
+                     ((reinterpret_cast<uintptr_t>(src1) & 15u) == 0);
+    const int64_t total = rows * a.ld_out / (vec ? 4 : 1);
+    int64_t blocks = (total + 256 * 2 - 1) / (256 * 2);
     const int64_t cap = (int64_t)ctx->sm_count * 8;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     KernelScope scope(ctx, SAMA_K_SPLIT, -1, st);
-    split_tf32_kernel<<<dim3((unsigned)blocks, 1, branches), 256, 0, st>>>(a);
+    if (vec)
+        split_tf32_kernel<true><<<dim3((unsigned)blocks, 1, branches), 256, 0, st>>>(a);
+    else
+        split_tf32_kernel<false><<<dim3((unsigned)blocks, 1, branches), 256, 0, st>>>(a);
     return cudaGetLastError();
 }
 
@@ -421,8 +447,10 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     // a box never exceeds the tensor's extent; rows of the shared-memory tile that no copy fills only
     // feed output rows / columns that the epilogue does not store
     const int a_box = L.M < BM ? L.M : BM, w_box = L.N < bn ? L.N : bn;
-    if (!make_map(&maps[0], L.a_hi, Kp, L.M, a_slabs, a_box) || !make_map(&maps[1], L.a_lo, Kp, L.M, a_slabs, a_box) ||
-        !make_map(&maps[2], L.w_hi, Kp, L.N, 2, w_box) || !make_map(&maps[3], L.w_lo, Kp, L.N, 2, w_box))
+    const int64_t a_slab = (int64_t)L.M * Kp;
+    if (!make_map(&maps[0], L.a_hi, Kp, L.M, a_slabs, a_box, a_slab) ||
+        !make_map(&maps[1], L.a_lo, Kp, L.M, a_slabs, a_box, a_slab) ||
+        !make_map(&maps[2], L.w_hi, Kp, L.N, 2, w_box, L.w_slab) || !make_map(&maps[3], L.w_lo, Kp, L.N, 2, w_box, L.w_slab))
         return cudaErrorInvalidValue;
     TcArgs a;
     a.bias[0] = L.bias[0];

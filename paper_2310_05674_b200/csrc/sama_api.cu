@@ -154,31 +154,53 @@ int validate_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, c
     return SAMA_OK;
 }
 
+SplitLayout make_split_layout(const sama_mlp_t* mlp) {
+    SplitLayout lay;
+    std::memset(&lay, 0, sizeof(lay));
+    lay.n_layers = mlp->n_layers;
+    int64_t off = 0, soff = 0;
+    for (int l = 0; l < mlp->n_layers; ++l) {
+        const int din = mlp->dims[l], dout = mlp->dims[l + 1];
+        lay.K[l] = din;
+        lay.Kp[l] = (din + 31) & ~31;
+        lay.w_off[l] = off;
+        lay.w_cnt[l] = (int64_t)din * dout;
+        lay.s_off[l] = soff;
+        off += (int64_t)din * dout + dout;
+        soff += (int64_t)dout * lay.Kp[l];
+    }
+    lay.slab = soff;
+    return lay;
+}
+
 // Whether this model fits the operand-split workspace of the tensor-core path.
 bool tc_fits(const sama_ctx* ctx, const sama_mlp_t* mlp, int32_t B) {
     auto r32 = [](int x) { return (size_t)((x + 31) & ~31); };
     const int L = mlp->n_layers;
     if (ctx->x_split_half == 0 || (size_t)B * r32(mlp->dims[0]) > ctx->x_split_half) return false;
-    for (int l = 0; l < L; ++l) {
-        if (2 * (size_t)mlp->dims[l + 1] * r32(mlp->dims[l]) > ctx->w_split_half) return false;
-        if (l + 1 < L && 2 * (size_t)B * r32(mlp->dims[l + 1]) > ctx->a_split_half) return false;
-    }
+    if (2 * (size_t)make_split_layout(mlp).slab > ctx->w_split_half) return false;
+    for (int l = 0; l + 1 < L; ++l)
+        if (2 * (size_t)B * r32(mlp->dims[l + 1]) > ctx->a_split_half) return false;
     return true;
 }
 
-// Forward pass of both branches on the tensor cores (3xTF32): operands are split into TF32 hi/lo
-// (X once, each layer's W+- before its product; hidden activations are split by the producing epilogue).
+// Forward pass of both branches on the tensor cores (3xTF32).  Operands are TF32 hi/lo pairs: X is split
+// here, hidden activations by the epilogue that produces them, and the weights either by the fused
+// perturbation sweep (w_presplit) or here, layer by layer.
 int run_forward_tc(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const float* theta_minus,
-                   const float* X, int32_t B, cudaStream_t st) {
+                   const float* X, int32_t B, bool w_presplit, cudaStream_t st) {
     const int L = mlp->n_layers;
-    SAMA_CUDA(ctx, launch_split_tf32(ctx, X, X, 1, B, mlp->dims[0], mlp->dims[0], ctx->x_split,
-                                     ctx->x_split + ctx->x_split_half, st));
-    int64_t off = 0;
+    const SplitLayout lay = make_split_layout(mlp);
+    float* w_hi = ctx->w_split;
+    float* w_lo = ctx->w_split + ctx->w_split_half;
+    SAMA_CUDA(ctx, launch_split_tf32(ctx, X, X, 1, B, mlp->dims[0], ctx->x_split, ctx->x_split + ctx->x_split_half,
+                                     0, st));
     for (int l = 0; l < L; ++l) {
         const int din = mlp->dims[l], dout = mlp->dims[l + 1];
         const bool last = (l + 1 == L);
-        SAMA_CUDA(ctx, launch_split_tf32(ctx, theta_plus + off, theta_minus + off, 2, dout, din, din, ctx->w_split,
-                                         ctx->w_split + ctx->w_split_half, st));
+        if (!w_presplit)
+            SAMA_CUDA(ctx, launch_split_tf32(ctx, theta_plus + lay.w_off[l], theta_minus + lay.w_off[l], 2, dout, din,
+                                             w_hi + lay.s_off[l], w_lo + lay.s_off[l], lay.slab, st));
         TcLayer t;
         if (l == 0) {
             t.a_hi = ctx->x_split;
@@ -187,10 +209,11 @@ int run_forward_tc(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus
             t.a_hi = ctx->a_split[(l - 1) & 1];
             t.a_lo = ctx->a_split[(l - 1) & 1] + ctx->a_split_half;
         }
-        t.w_hi = ctx->w_split;
-        t.w_lo = ctx->w_split + ctx->w_split_half;
-        t.bias[0] = theta_plus + off + (int64_t)din * dout;
-        t.bias[1] = theta_minus + off + (int64_t)din * dout;
+        t.w_hi = w_hi + lay.s_off[l];
+        t.w_lo = w_lo + lay.s_off[l];
+        t.w_slab = lay.slab;
+        t.bias[0] = theta_plus + lay.w_off[l] + lay.w_cnt[l];
+        t.bias[1] = theta_minus + lay.w_off[l] + lay.w_cnt[l];
         t.out_f32[0] = ctx->logits;
         t.out_f32[1] = ctx->logits + (int64_t)B * dout;
         t.out_hi = last ? nullptr : ctx->a_split[l & 1];
@@ -204,7 +227,6 @@ int run_forward_tc(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus
         t.shared_a = (l == 0) ? 1 : 0;
         t.layer = l;
         SAMA_CUDA(ctx, launch_gemm_tf32x3(ctx, t, st));
-        off += (int64_t)din * dout + dout;
     }
     return SAMA_OK;
 }
@@ -212,13 +234,14 @@ int run_forward_tc(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus
 // The dual-branch forward and the finite difference, arguments already validated.
 int run_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const float* theta_minus,
            const float* X, const int32_t* y, const float* lambda, int32_t B, const float* eps_fd,
-           float* metagrad_out, float* loss_plus_out, float* loss_minus_out, cudaStream_t st) {
+           float* metagrad_out, float* loss_plus_out, float* loss_minus_out, cudaStream_t st,
+           bool w_presplit = false) {
     const int L = mlp->n_layers;
     const int C = mlp->dims[L];
     const bool fits = tc_fits(ctx, mlp, B);
     if (ctx->gemm_mode == 2 && !fits) return SAMA_ERR_SIZE;
     if (ctx->gemm_mode != 1 && fits) {
-        const int rc = run_forward_tc(ctx, mlp, theta_plus, theta_minus, X, B, st);
+        const int rc = run_forward_tc(ctx, mlp, theta_plus, theta_minus, X, B, w_presplit, st);
         if (rc != SAMA_OK) return rc;
         SAMA_CUDA(ctx, launch_ce_fd(ctx, ctx->logits, ctx->logits + (int64_t)B * C, C, y, lambda, B, C,
                                     eps_fd ? eps_fd : &ctx->scalars->eps_fd, metagrad_out, loss_plus_out,
@@ -318,14 +341,13 @@ int sama_create(sama_ctx** out, int device, int64_t max_n, int32_t max_batch, co
         ok = ok && cudaMalloc(&ctx->logits, sizeof(float) * 2 * (size_t)max_batch * ctx->max_classes) == cudaSuccess;
         // operand splits of the tensor-core path
         auto r32 = [](int x) { return (size_t)((x + 31) & ~31); };
-        size_t wmax = 0, amax = 0;
-        for (int l = 0; l < L; ++l) {
-            const size_t we = (size_t)mlp->dims[l + 1] * r32(mlp->dims[l]);
-            wmax = we > wmax ? we : wmax;
-            if (l + 1 < L) { const size_t ae = r32(mlp->dims[l + 1]); amax = ae > amax ? ae : amax; }
+        size_t amax = 0;
+        for (int l = 0; l + 1 < L; ++l) {
+            const size_t ae = r32(mlp->dims[l + 1]);
+            amax = ae > amax ? ae : amax;
         }
         ctx->x_split_half = (size_t)max_batch * r32(mlp->dims[0]);
-        ctx->w_split_half = 2 * wmax;
+        ctx->w_split_half = 2 * (size_t)make_split_layout(mlp).slab;
         ctx->a_split_half = 2 * (size_t)max_batch * amax;
         ok = ok && cudaMalloc(&ctx->x_split, sizeof(float) * 2 * ctx->x_split_half) == cudaSuccess &&
              cudaMalloc(&ctx->w_split, sizeof(float) * 2 * ctx->w_split_half) == cudaSuccess;
@@ -441,10 +463,19 @@ int sama_step(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* thet
     if (!guard.ok) return SAMA_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;
     SAMA_CUDA(ctx, launch_adapt_sumsq(ctx, n, m, s, c.identity ? nullptr : g_base, g_meta, c, p_out, nullptr, st));
-    SAMA_CUDA(ctx, launch_perturb(ctx, n, theta, p_out, &ctx->scalars->sumsq, alpha, theta_plus, theta_minus,
-                                  nullptr, st));
+    // With the tensor-core forward, the perturbation sweep also emits the TF32 operand split of W+-.
+    const SplitLayout lay = make_split_layout(mlp);
+    const bool fused = ctx->gemm_mode != 1 && tc_fits(ctx, mlp, B) &&
+                       perturb_split_applicable(lay, theta, p_out, theta_plus, theta_minus);
+    if (fused)
+        SAMA_CUDA(ctx, launch_perturb_split(ctx, n, theta, p_out, &ctx->scalars->sumsq, alpha, theta_plus,
+                                            theta_minus, nullptr, lay, ctx->w_split,
+                                            ctx->w_split + ctx->w_split_half, st));
+    else
+        SAMA_CUDA(ctx, launch_perturb(ctx, n, theta, p_out, &ctx->scalars->sumsq, alpha, theta_plus, theta_minus,
+                                      nullptr, st));
     return run_fd(ctx, mlp, theta_plus, theta_minus, X, y, lambda, B, nullptr, metagrad_out, loss_plus_out,
-                  loss_minus_out, st);
+                  loss_minus_out, st, fused);
 }
 
 int sama_step_host(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* theta_host, const float* m_host,

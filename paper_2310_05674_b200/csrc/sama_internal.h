@@ -33,6 +33,17 @@ struct AdaptConsts {
     int identity;
 };
 
+// Where each layer's weight matrix lives in the flat parameter vector and in one
+// branch slab of the TF32 hi/lo split buffers (rows padded to a multiple of 32).
+struct SplitLayout {
+    int n_layers;
+    int32_t K[kMaxLayers], Kp[kMaxLayers];
+    int64_t w_off[kMaxLayers];  // offset of W_l in theta
+    int64_t w_cnt[kMaxLayers];  // d_l * d_{l-1}
+    int64_t s_off[kMaxLayers];  // offset of layer l inside a slab
+    int64_t slab;               // floats per slab = sum_l d_l * Kp_l
+};
+
 struct ProfRecord {
     int kind, layer;
     cudaEvent_t start, stop;
@@ -60,7 +71,7 @@ struct sama_ctx {
     float* logits;                 // device [2][max_batch][max_classes]
     // TF32 hi/lo operand splits of the tensor-core path, each buffer holds hi then lo
     float* x_split;                // device [2][max_batch][round32(d_0)]
-    float* w_split;                // device [2][2][max_l d_l round32(d_{l-1})]
+    float* w_split;                // device [hi, lo][2 branches][slab]: every layer's W, rows padded to 32
     float* a_split[2];             // device, ping-pong: [2][2][max_batch][round32(max hidden)]
     size_t x_split_half, w_split_half, a_split_half;  // floats per hi (or lo) part; 0 = path unavailable
     float* stage;                  // device: staging of the host entry point (allocated on first use)
@@ -103,6 +114,12 @@ cudaError_t launch_adapt_sumsq(sama_ctx* ctx, int64_t n, const float* m, const f
 cudaError_t launch_sumsq(sama_ctx* ctx, int64_t n, const float* p, cudaStream_t st);
 cudaError_t launch_perturb(sama_ctx* ctx, int64_t n, const float* theta, const float* p, const double* sumsq,
                            float alpha, float* theta_plus, float* theta_minus, float* eps_fd_out, cudaStream_t st);
+// perturb that also writes the TF32 hi/lo split of every weight matrix of theta+ and theta- (same sweep)
+bool perturb_split_applicable(const SplitLayout& lay, const float* theta, const float* p, const float* theta_plus,
+                              const float* theta_minus);
+cudaError_t launch_perturb_split(sama_ctx* ctx, int64_t n, const float* theta, const float* p, const double* sumsq,
+                                 float alpha, float* theta_plus, float* theta_minus, float* eps_fd_out,
+                                 const SplitLayout& lay, float* hi, float* lo, cudaStream_t st);
 
 // One layer of both branches: C[b] = act(A[b] * W[b]^T + bias[b]) for b in {0, 1}
 struct GemmArgs {
@@ -124,8 +141,9 @@ cudaError_t launch_gemm(sama_ctx* ctx, const GemmArgs& g, cudaStream_t st);
 struct TcLayer {
     const float* a_hi;     // [shared_a ? 1 : 2][M][round32(K)]
     const float* a_lo;
-    const float* w_hi;     // [2][N][round32(K)]
+    const float* w_hi;     // [2][N][round32(K)], branch b at w_hi + b * w_slab
     const float* w_lo;
+    int64_t w_slab;
     const float* bias[2];  // [N]
     float* out_f32[2];     // last layer: [M][ldc]
     float* out_hi;         // hidden layers: [2][M][round32(N)]
@@ -134,7 +152,7 @@ struct TcLayer {
     int relu, last, shared_a, layer;
 };
 cudaError_t launch_split_tf32(sama_ctx* ctx, const float* src0, const float* src1, int branches, int64_t rows,
-                              int cols, int ld_src, float* hi, float* lo, cudaStream_t st);
+                              int cols, float* hi, float* lo, int64_t slab, cudaStream_t st);
 cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st);
 
 // ce_fd.cu
