@@ -139,7 +139,7 @@ __device__ __forceinline__ float to_tf32(float x) {
 
 struct TcArgs {
     const float* bias[2];  // [N] fp32 (slices of theta+ / theta-), may be unaligned
-    float* out_f32[2];     // last layer: logits [M][ldc]
+    float* out_f32[2];     // fp32 output (logits, or activations feeding a fused head): [M][ldc]
     float* out_hi;         // hidden layers: next operand hi, [2][M][ld_next]
     float* out_lo;
     int M, N, num_kb;
@@ -277,9 +277,16 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                     }
                     if (args.last) {
                         float* dst = (br ? args.out_f32[1] : args.out_f32[0]) + (int64_t)m * args.ldc + n;
+                        if (n + 15 < args.N && (args.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (n + j < args.N) dst[j] = v[j];
+                            for (int j = 0; j < 4; ++j)
+                                reinterpret_cast<float4*>(dst)[j] =
+                                    make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (n + j < args.N) dst[j] = v[j];
+                        }
                     } else if (n < args.ld_next) {
                         // columns in [N, ld_next) are the next layer's zero padding along K
                         const int64_t off = ((int64_t)br * args.M + m) * args.ld_next + n;
@@ -441,7 +448,8 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     // N-tile: 16 for a narrow last layer; 64 when 128-wide tiles would leave SMs idle; else 128.
     // (Hidden layers never take 16: their tiles must also write the zero padding up to round_up32(N).)
     const int64_t tiles128 = (int64_t)((L.M + BM - 1) / BM) * ((L.N + 127) / 128) * 2;
-    const int bn = (L.last && L.N <= 16) ? 16 : ((L.N <= 64 || tiles128 < ctx->sm_count) ? 64 : 128);
+    int bn = (L.last && L.N <= 16) ? 16 : ((L.N <= 64 || tiles128 < ctx->sm_count) ? 64 : 128);
+    if (ctx->tile_override == 64 || ctx->tile_override == 128) bn = ctx->tile_override;
     CUtensorMap maps[4];
     const int a_slabs = L.shared_a ? 1 : 2;
     // a box never exceeds the tensor's extent; rows of the shared-memory tile that no copy fills only

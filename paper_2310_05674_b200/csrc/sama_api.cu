@@ -188,8 +188,12 @@ bool tc_fits(const sama_ctx* ctx, const sama_mlp_t* mlp, int32_t B) {
 // here, hidden activations by the epilogue that produces them, and the weights either by the fused
 // perturbation sweep (w_presplit) or here, layer by layer.
 int run_forward_tc(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const float* theta_minus,
-                   const float* X, int32_t B, bool w_presplit, cudaStream_t st) {
-    const int L = mlp->n_layers;
+                   const float* X, int32_t B, bool w_presplit, bool fused_head, cudaStream_t st) {
+    // with a fused head the last layer is not a matrix product here, and the layer before it
+    // leaves fp32 activations (ReLU applied) in the context's activation buffer
+    const int L = fused_head ? mlp->n_layers - 1 : mlp->n_layers;
+    if (L == 0) return SAMA_OK;
+    float* f32_out = fused_head ? ctx->act[0] : ctx->logits;
     const SplitLayout lay = make_split_layout(mlp);
     float* w_hi = ctx->w_split;
     float* w_lo = ctx->w_split + ctx->w_split_half;
@@ -214,15 +218,15 @@ int run_forward_tc(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus
         t.w_slab = lay.slab;
         t.bias[0] = theta_plus + lay.w_off[l] + lay.w_cnt[l];
         t.bias[1] = theta_minus + lay.w_off[l] + lay.w_cnt[l];
-        t.out_f32[0] = ctx->logits;
-        t.out_f32[1] = ctx->logits + (int64_t)B * dout;
+        t.out_f32[0] = f32_out;
+        t.out_f32[1] = f32_out + (int64_t)B * dout;
         t.out_hi = last ? nullptr : ctx->a_split[l & 1];
         t.out_lo = last ? nullptr : ctx->a_split[l & 1] + ctx->a_split_half;
         t.M = B;
         t.N = dout;
         t.K = din;
         t.ldc = dout;
-        t.relu = last ? 0 : 1;
+        t.relu = (last && !fused_head) ? 0 : 1;
         t.last = last ? 1 : 0;
         t.shared_a = (l == 0) ? 1 : 0;
         t.layer = l;
@@ -240,46 +244,63 @@ int run_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const 
     const int C = mlp->dims[L];
     const bool fits = tc_fits(ctx, mlp, B);
     if (ctx->gemm_mode == 2 && !fits) return SAMA_ERR_SIZE;
-    if (ctx->gemm_mode != 1 && fits) {
-        const int rc = run_forward_tc(ctx, mlp, theta_plus, theta_minus, X, B, w_presplit, st);
-        if (rc != SAMA_OK) return rc;
-        SAMA_CUDA(ctx, launch_ce_fd(ctx, ctx->logits, ctx->logits + (int64_t)B * C, C, y, lambda, B, C,
-                                    eps_fd ? eps_fd : &ctx->scalars->eps_fd, metagrad_out, loss_plus_out,
-                                    loss_minus_out, st));
-        return SAMA_OK;
-    }
-    const float* in[2] = {X, X};
+    const bool use_tc = ctx->gemm_mode != 1 && fits;
+    const bool fused_head = head_applicable(C);
+    const float* eps = eps_fd ? eps_fd : &ctx->scalars->eps_fd;
+    const int n_gemm = fused_head ? L - 1 : L;  // layers computed as matrix products
+    const float* in[2] = {X, X};                // fp32 input of the next stage
     int ld_in = mlp->dims[0];
-    int64_t off = 0;
-    for (int l = 0; l < L; ++l) {
-        const int din = mlp->dims[l], dout = mlp->dims[l + 1];
-        const bool last = (l + 1 == L);
-        float* out0 = last ? ctx->logits : ctx->act[l & 1];
-        GemmArgs g;
-        g.A[0] = in[0];
-        g.A[1] = in[1];
-        g.W[0] = theta_plus + off;
-        g.W[1] = theta_minus + off;
-        g.bias[0] = theta_plus + off + (int64_t)din * dout;
-        g.bias[1] = theta_minus + off + (int64_t)din * dout;
-        g.C[0] = out0;
-        g.C[1] = out0 + (int64_t)B * dout;
-        g.M = B;
-        g.N = dout;
-        g.K = din;
-        g.lda = ld_in;
-        g.ldw = din;
-        g.ldc = dout;
-        g.relu = last ? 0 : 1;
-        g.layer = l;
-        SAMA_CUDA(ctx, launch_gemm(ctx, g, st));
-        in[0] = g.C[0];
-        in[1] = g.C[1];
-        ld_in = dout;
-        off += (int64_t)din * dout + dout;
+
+    if (use_tc) {
+        const int rc = run_forward_tc(ctx, mlp, theta_plus, theta_minus, X, B, w_presplit, fused_head, st);
+        if (rc != SAMA_OK) return rc;
+        if (n_gemm > 0) {
+            float* out = fused_head ? ctx->act[0] : ctx->logits;
+            in[0] = out;
+            in[1] = out + (int64_t)B * mlp->dims[n_gemm];
+            ld_in = mlp->dims[n_gemm];
+        }
+    } else {
+        int64_t off = 0;
+        for (int l = 0; l < n_gemm; ++l) {
+            const int din = mlp->dims[l], dout = mlp->dims[l + 1];
+            const bool last = (l + 1 == L);
+            float* out0 = last ? ctx->logits : ctx->act[l & 1];
+            GemmArgs g;
+            g.A[0] = in[0];
+            g.A[1] = in[1];
+            g.W[0] = theta_plus + off;
+            g.W[1] = theta_minus + off;
+            g.bias[0] = theta_plus + off + (int64_t)din * dout;
+            g.bias[1] = theta_minus + off + (int64_t)din * dout;
+            g.C[0] = out0;
+            g.C[1] = out0 + (int64_t)B * dout;
+            g.M = B;
+            g.N = dout;
+            g.K = din;
+            g.lda = ld_in;
+            g.ldw = din;
+            g.ldc = dout;
+            g.relu = last ? 0 : 1;
+            g.layer = l;
+            SAMA_CUDA(ctx, launch_gemm(ctx, g, st));
+            in[0] = g.C[0];
+            in[1] = g.C[1];
+            ld_in = dout;
+            off += (int64_t)din * dout + dout;
+        }
     }
-    SAMA_CUDA(ctx, launch_ce_fd(ctx, in[0], in[1], C, y, lambda, B, C, eps_fd ? eps_fd : &ctx->scalars->eps_fd,
-                                metagrad_out, loss_plus_out, loss_minus_out, st));
+    if (fused_head) {
+        int64_t off = 0;
+        for (int l = 0; l + 1 < L; ++l) off += (int64_t)mlp->dims[l] * mlp->dims[l + 1] + mlp->dims[l + 1];
+        const int K = mlp->dims[L - 1];
+        SAMA_CUDA(ctx, launch_head_ce_fd(ctx, in[0], in[1], ld_in, theta_plus + off, theta_minus + off,
+                                         theta_plus + off + (int64_t)K * C, theta_minus + off + (int64_t)K * C, y,
+                                         lambda, B, C, K, eps, metagrad_out, loss_plus_out, loss_minus_out, st));
+    } else {
+        SAMA_CUDA(ctx, launch_ce_fd(ctx, in[0], in[1], C, y, lambda, B, C, eps, metagrad_out, loss_plus_out,
+                                    loss_minus_out, st));
+    }
     return SAMA_OK;
 }
 
@@ -325,6 +346,7 @@ int sama_create(sama_ctx** out, int device, int64_t max_n, int32_t max_batch, co
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return SAMA_ERR_CUDA; }
     ctx->sm_count = prop.multiProcessorCount;
+    if (const char* t = std::getenv("SAMA_TC_TILE")) ctx->tile_override = std::atoi(t);
     bool ok = cudaMalloc(&ctx->scalars, sizeof(DeviceScalars)) == cudaSuccess &&
               cudaMemset(ctx->scalars, 0, sizeof(DeviceScalars)) == cudaSuccess &&
               cudaMalloc(&ctx->partials, sizeof(double) * kMaxPartials) == cudaSuccess;

@@ -63,6 +63,7 @@ struct sama_ctx {
     int32_t max_width;    // widest hidden layer the forward workspace covers, 0 if none
     int32_t max_classes;  // largest d_L covered, 0 if the context has no forward workspace
     int gemm_mode;        // 0 auto, 1 ffma, 2 3xTF32
+    int tile_override;    // 0, or an N-tile width forced through the SAMA_TC_TILE environment variable (tuning aid)
     int last_cuda_error;
     int64_t launches;
     sama::DeviceScalars* scalars;  // device
@@ -159,5 +160,12 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
 cudaError_t launch_ce_fd(sama_ctx* ctx, const float* z_plus, const float* z_minus, int ldz, const int32_t* y,
                          const float* lambda, int B, int C, const float* eps_fd, float* metagrad,
                          float* loss_plus, float* loss_minus, cudaStream_t st);
+
+// head_ce_fd.cu : narrow last layer (C <= 16) + cross-entropy + central difference in one kernel
+bool head_applicable(int C);
+cudaError_t launch_head_ce_fd(sama_ctx* ctx, const float* h_plus, const float* h_minus, int ldh,
+                              const float* w_plus, const float* w_minus, const float* b_plus, const float* b_minus,
+                              const int32_t* y, const float* lambda, int B, int C, int K, const float* eps_fd,
+                              float* metagrad, float* loss_plus, float* loss_minus, cudaStream_t st);
 
 }  // namespace sama
