@@ -28,6 +28,8 @@
 // bounded) for the copies it has in flight, frees its tensor memory and exits.
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include "sama_internal.h"
 
 namespace sama {
@@ -145,6 +147,7 @@ struct TcArgs {
     int M, N, num_kb;
     int ldc, ld_next;      // ld_next = N rounded up to 32 (zero-filled tail)
     int relu, last, shared_a;
+    int tiles_m, tiles_n, group_n;
     uint32_t tx_bytes;     // bytes the four copies of one k-block deliver
     int32_t* status;
 };
@@ -175,7 +178,18 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int br = blockIdx.z;
-    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    // Tile order: CTAs that run together cover all M-tiles of a group of `group_n` N-tiles, so one wave
+    // re-uses a bounded set of W tiles and every A tile from L2 instead of sweeping all of W.
+    int tile_m, tile_n;
+    {
+        const int per_group = args.group_n * args.tiles_m;
+        const int group = blockIdx.x / per_group, rem = blockIdx.x - group * per_group;
+        const int first_n = group * args.group_n;
+        const int gsz = min(args.group_n, args.tiles_n - first_n);
+        tile_n = first_n + rem % gsz;
+        tile_m = rem / gsz;
+    }
+    const int m0 = tile_m * BM, n0 = tile_n * BN;
     const int num_kb = args.num_kb;
 
     if (threadIdx.x == 0) {
@@ -477,7 +491,14 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     a.shared_a = L.shared_a;
     a.tx_bytes = (uint32_t)(2 * a_box * BKF * 4 + 2 * w_box * BKF * 4);
     a.status = &ctx->scalars->status;
-    dim3 grid((L.N + bn - 1) / bn, (L.M + BM - 1) / BM, 2);
+    a.tiles_m = (L.M + BM - 1) / BM;
+    a.tiles_n = (L.N + bn - 1) / bn;
+    // about one wave of CTAs per group: group_n N-tiles x all M-tiles
+    a.group_n = ctx->sm_count / a.tiles_m;
+    if (a.group_n < 1) a.group_n = 1;
+    if (a.group_n > a.tiles_n) a.group_n = a.tiles_n;
+    if (const char* e = std::getenv("SAMA_TC_GROUP")) { const int g = std::atoi(e); if (g >= 1 && g <= a.tiles_n) a.group_n = g; }
+    dim3 grid(a.tiles_m * a.tiles_n, 1, 2);
     KernelScope scope(ctx, SAMA_K_GEMM_TF32X3, L.layer, st);
     if (bn == 16) return launch_tc<16>(maps, a, grid, st);
     if (bn == 64) return launch_tc<64>(maps, a, grid, st);
