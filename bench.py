@@ -105,6 +105,7 @@ def source_hash(*names):
 
 
 KERNEL_SOURCES = {"adapt_sumsq": ("adapt_perturb.cu",), "perturb": ("adapt_perturb.cu",), "sumsq": ("adapt_perturb.cu",),
+                  "perturb_split": ("adapt_perturb.cu",), "head_ce_fd": ("head_ce_fd.cu",),
                   "gemm_ffma": ("gemm_ffma.cu",), "ce_fd": ("ce_fd.cu",), "gemm_tf32x3": ("gemm_tf32x3.cu",),
                   "split_tf32": ("gemm_tf32x3.cu",)}
 
@@ -349,6 +350,8 @@ def main():
         rooflines["adapt_sumsq"] = hbm_roof("adapt_sumsq", 20.0 * n)
     if "perturb" in per_kernel:
         rooflines["perturb"] = hbm_roof("perturb", 16.0 * n)
+    if "perturb_split" in per_kernel:  # perturb + TF32 hi/lo of both branches: 8 read + 8 + 16 written per element
+        rooflines["perturb_split"] = hbm_roof("perturb_split", 32.0 * n)
     for gk in ("gemm_ffma", "gemm_tf32x3"):
         if gk in per_kernel and cfg:
             flops = float(cfg.forward_flops)

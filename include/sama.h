@@ -225,7 +225,8 @@ enum {
     SAMA_K_CE_FD = 4,
     SAMA_K_SPLIT = 5,
     SAMA_K_GEMM_TF32X3 = 6,
-    SAMA_K_HEAD = 7 /* narrow last layer fused with cross-entropy + central difference */
+    SAMA_K_HEAD = 7, /* narrow last layer fused with cross-entropy + central difference */
+    SAMA_K_PERTURB_SPLIT = 8 /* perturbation that also writes the tensor-core operands of W+ and W- */
 };
 typedef struct sama_kernel_time_t {
     int32_t kind;  /* SAMA_K_* */

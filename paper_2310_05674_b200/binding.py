@@ -47,7 +47,7 @@ class sama_kernel_time_t(C.Structure):
 
 
 KERNEL_KINDS = {0: "adapt_sumsq", 1: "sumsq", 2: "perturb", 3: "gemm_ffma", 4: "ce_fd", 5: "split_tf32",
-                6: "gemm_tf32x3", 7: "head_ce_fd"}
+                6: "gemm_tf32x3", 7: "head_ce_fd", 8: "perturb_split"}
 
 
 class sama_mlp_t(C.Structure):

@@ -430,7 +430,7 @@ bool perturb_split_applicable(const SplitLayout& lay, const float* theta, const 
 cudaError_t launch_perturb_split(sama_ctx* ctx, int64_t n, const float* theta, const float* p, const double* sumsq,
                                  float alpha, float* theta_plus, float* theta_minus, float* eps_fd_out,
                                  const SplitLayout& lay, float* hi, float* lo, cudaStream_t st) {
-    KernelScope scope(ctx, SAMA_K_PERTURB, -1, st);
+    KernelScope scope(ctx, SAMA_K_PERTURB_SPLIT, -1, st);
     perturb_split_kernel<<<stream_grid(ctx, n >> 2, kUnroll), kThreads, 0, st>>>(
         n, theta, p, sumsq, alpha, theta_plus, theta_minus, ctx->scalars, eps_fd_out, lay, hi, lo);
     return cudaGetLastError();

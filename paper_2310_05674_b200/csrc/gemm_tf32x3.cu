@@ -148,6 +148,9 @@ struct TcArgs {
     int ldc, ld_next;      // ld_next = N rounded up to 32 (zero-filled tail)
     int relu, last, shared_a;
     int tiles_m, tiles_n, group_n;
+    int splits, kb_per_split;  // split-K: grid.z = 2 * splits, each CTA takes kb_per_split k-blocks
+    float* ws;                 // split-K partial tiles [2 * tiles][splits][BM][BN]
+    int* counters;             // split-K arrival counters [2 * tiles], zero between launches
     uint32_t tx_bytes;     // bytes the four copies of one k-block deliver
     int32_t* status;
 };
@@ -176,8 +179,12 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     volatile uint32_t* tmem_ptr_slot =
         reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
 
+    const uint32_t last_slot = abort_slot + 4;
+    volatile uint32_t* last_flag =
+        reinterpret_cast<volatile uint32_t*>(smem_raw + (last_slot - smem_u32(smem_raw)));
+
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int br = blockIdx.z;
+    const int br = blockIdx.z / args.splits, split = blockIdx.z - br * args.splits;
     // Tile order: CTAs that run together cover all M-tiles of a group of `group_n` N-tiles, so one wave
     // re-uses a bounded set of W tiles and every A tile from L2 instead of sweeping all of W.
     int tile_m, tile_n;
@@ -190,7 +197,9 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         tile_m = rem / gsz;
     }
     const int m0 = tile_m * BM, n0 = tile_n * BN;
-    const int num_kb = args.num_kb;
+    // this CTA's share of the contraction (the host guarantees at least one k-block per split)
+    const int kb_begin = split * args.kb_per_split;
+    const int num_kb = min(args.kb_per_split, args.num_kb - kb_begin);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -224,10 +233,11 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                 if (*abort_flag) break;
                 const uint32_t st = base + s * STAGE;
                 mbar_expect_tx(full_bar(s), args.tx_bytes);
-                tma_load_3d(st, &map_a_hi, full_bar(s), kb * BKF, m0, za);
-                tma_load_3d(st + A_BYTES, &map_a_lo, full_bar(s), kb * BKF, m0, za);
-                tma_load_3d(st + 2 * A_BYTES, &map_w_hi, full_bar(s), kb * BKF, n0, br);
-                tma_load_3d(st + 2 * A_BYTES + W_BYTES, &map_w_lo, full_bar(s), kb * BKF, n0, br);
+                const int kx = (kb_begin + kb) * BKF;
+                tma_load_3d(st, &map_a_hi, full_bar(s), kx, m0, za);
+                tma_load_3d(st + A_BYTES, &map_a_lo, full_bar(s), kx, m0, za);
+                tma_load_3d(st + 2 * A_BYTES, &map_w_hi, full_bar(s), kx, n0, br);
+                tma_load_3d(st + 2 * A_BYTES + W_BYTES, &map_w_lo, full_bar(s), kx, n0, br);
                 issued = kb + 1;
             }
             if (*abort_flag) {
@@ -272,15 +282,64 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
             }
         }
         ok = __shfl_sync(0xffffffffu, ok, 0);
+        // the four epilogue warps proceed together or not at all (they meet again at named barrier 1)
+        volatile uint32_t* ok_slots = last_flag + 1;
+        if (lane == 0) ok_slots[q] = ok ? 1u : 0u;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        ok = (ok_slots[0] & ok_slots[1] & ok_slots[2] & ok_slots[3]) != 0;
         if (ok) {
             tc_fence_after();
-            const int m = m0 + q * 32 + lane;
+            const int row = q * 32 + lane;
+            const int m = m0 + row;
             const float* bias = br ? args.bias[1] : args.bias[0];
             const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+            // Split-K: every CTA of a tile stores its raw partial; the last one to arrive adds the
+            // partials in split order (so the sum does not depend on which CTA that is) and finishes.
+            const float* part = nullptr;
+            bool finish = true;
+            if (args.splits > 1) {
+                const int tile_lin = br * (args.tiles_m * args.tiles_n) + (int)blockIdx.x;
+                float* base_ws = args.ws + (int64_t)tile_lin * args.splits * (BM * BN);
+                float* mine = base_ws + ((int64_t)split * BM + row) * BN;
 #pragma unroll 1
-            for (int c = 0; c < BN; c += 16) {
+                for (int c = 0; c < BN; c += 16) {
+                    float v[16];
+                    tmem_ld16(lane_addr + c, v);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        __stcg(reinterpret_cast<float4*>(mine + c) + j,
+                               make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]));
+                }
+                __threadfence();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (warp == 2 && lane == 0) {
+                    const int prev = atomicAdd(args.counters + tile_lin, 1);
+                    const bool is_last = (prev == args.splits - 1);
+                    if (is_last) args.counters[tile_lin] = 0;  // every CTA of the tile has arrived
+                    *last_flag = is_last ? 1u : 0u;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                finish = (*last_flag != 0);
+                if (finish) __threadfence();
+                part = base_ws + (int64_t)row * BN;
+            }
+#pragma unroll 1
+            for (int c = 0; finish && c < BN; c += 16) {
                 float v[16];
-                tmem_ld16(lane_addr + c, v);   // all lanes take part (sync.aligned)
+                if (part) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] = 0.f;
+                    for (int sp = 0; sp < args.splits; ++sp) {
+                        const float4* src = reinterpret_cast<const float4*>(part + (int64_t)sp * (BM * BN) + c);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float4 t = __ldcg(src + j);
+                            v[4 * j] += t.x; v[4 * j + 1] += t.y; v[4 * j + 2] += t.z; v[4 * j + 3] += t.w;
+                        }
+                    }
+                } else {
+                    tmem_ld16(lane_addr + c, v);   // all lanes take part (sync.aligned)
+                }
                 const int n = n0 + c;
                 if (m < args.M) {
 #pragma unroll
@@ -462,8 +521,24 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     // N-tile: 16 for a narrow last layer; 64 when 128-wide tiles would leave SMs idle; else 128.
     // (Hidden layers never take 16: their tiles must also write the zero padding up to round_up32(N).)
     const int64_t tiles128 = (int64_t)((L.M + BM - 1) / BM) * ((L.N + 127) / 128) * 2;
-    int bn = (L.last && L.N <= 16) ? 16 : ((L.N <= 64 || tiles128 < ctx->sm_count) ? 64 : 128);
+    // When even that leaves SMs idle the contraction is split over several CTAs per tile (split-K).
+    const bool narrow_last = L.last && L.N <= 16;
+    int bn = narrow_last ? 16 : (L.N <= 64 ? 64 : 128);
     if (ctx->tile_override == 64 || ctx->tile_override == 128) bn = ctx->tile_override;
+    const int num_kb_total = Kp / BKF;
+    int splits = 1;
+    {
+        const int64_t tiles = (int64_t)((L.M + BM - 1) / BM) * ((L.N + bn - 1) / bn) * 2;
+        int want = (int)(ctx->sm_count / (tiles > 0 ? tiles : 1));
+        if (const char* e = std::getenv("SAMA_TC_SPLITS")) want = std::atoi(e);
+        if (want > 8) want = 8;
+        const int by_k = num_kb_total / 4;  // at least 4 k-blocks per split
+        if (want > by_k) want = by_k;
+        while (want > 1 && (size_t)tiles * want * BM * bn > ctx->tc_ws_floats) --want;
+        if (tiles > kTcCounters) want = 1;
+        if (want > 1 && ctx->tc_ws && ctx->tc_counters) splits = want;
+    }
+    (void)tiles128;
     CUtensorMap maps[4];
     const int a_slabs = L.shared_a ? 1 : 2;
     // a box never exceeds the tensor's extent; rows of the shared-memory tile that no copy fills only
@@ -494,11 +569,15 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     a.tiles_m = (L.M + BM - 1) / BM;
     a.tiles_n = (L.N + bn - 1) / bn;
     // about one wave of CTAs per group: group_n N-tiles x all M-tiles
+    a.kb_per_split = (num_kb_total + splits - 1) / splits;
+    a.splits = (num_kb_total + a.kb_per_split - 1) / a.kb_per_split;  // no empty split
+    a.ws = ctx->tc_ws;
+    a.counters = ctx->tc_counters;
     a.group_n = ctx->sm_count / a.tiles_m;
     if (a.group_n < 1) a.group_n = 1;
     if (a.group_n > a.tiles_n) a.group_n = a.tiles_n;
     if (const char* e = std::getenv("SAMA_TC_GROUP")) { const int g = std::atoi(e); if (g >= 1 && g <= a.tiles_n) a.group_n = g; }
-    dim3 grid(a.tiles_m * a.tiles_n, 1, 2);
+    dim3 grid(a.tiles_m * a.tiles_n, 1, 2 * a.splits);
     KernelScope scope(ctx, SAMA_K_GEMM_TF32X3, L.layer, st);
     if (bn == 16) return launch_tc<16>(maps, a, grid, st);
     if (bn == 64) return launch_tc<64>(maps, a, grid, st);

@@ -373,6 +373,10 @@ int sama_create(sama_ctx** out, int device, int64_t max_n, int32_t max_batch, co
         ctx->a_split_half = 2 * (size_t)max_batch * amax;
         ok = ok && cudaMalloc(&ctx->x_split, sizeof(float) * 2 * ctx->x_split_half) == cudaSuccess &&
              cudaMalloc(&ctx->w_split, sizeof(float) * 2 * ctx->w_split_half) == cudaSuccess;
+        ctx->tc_ws_floats = (size_t)8 << 20;  // 32 MiB of split-K partial tiles
+        ok = ok && cudaMalloc(&ctx->tc_ws, sizeof(float) * ctx->tc_ws_floats) == cudaSuccess &&
+             cudaMalloc(&ctx->tc_counters, sizeof(int) * kTcCounters) == cudaSuccess &&
+             cudaMemset(ctx->tc_counters, 0, sizeof(int) * kTcCounters) == cudaSuccess;
         if (ok && amax > 0)
             ok = cudaMalloc(&ctx->a_split[0], sizeof(float) * 2 * ctx->a_split_half) == cudaSuccess &&
                  cudaMalloc(&ctx->a_split[1], sizeof(float) * 2 * ctx->a_split_half) == cudaSuccess;
@@ -398,6 +402,8 @@ int sama_destroy(sama_ctx* ctx) {
     cudaFree(ctx->w_split);
     cudaFree(ctx->a_split[0]);
     cudaFree(ctx->a_split[1]);
+    cudaFree(ctx->tc_ws);
+    cudaFree(ctx->tc_counters);
     cudaFree(ctx->stage);
     if (ctx->prof) {
         for (auto& r : ctx->prof->records) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }

@@ -273,6 +273,19 @@ def test_step_parity_wide4096_sampled(gemm_mode):
     check_step(cfg, w, B.Adam(), 1.0, rows=rows[::2], gemm_mode=gemm_mode, key=("wide4096", 1.0))
 
 
+@pytest.mark.parametrize("gemm_mode", GEMM_MODES)
+def test_step_is_bitwise_reproducible(gemm_mode):
+    """Fixed reduction orders everywhere (norm partials, split-K partial tiles): repeated steps agree bit for bit."""
+    for cfg, w in [(W.CONFIGS["tiny"], W.mlp_workload(W.CONFIGS["tiny"], 0)), W.custom_mlp((40, 200, 72, 24), 257, seed=5),
+                   W.custom_mlp((2048, 512, 40), 256, seed=6)]:
+        with Ctx(cfg.n_params, cfg.batch, cfg.dims, gemm_mode) as ctx:
+            runs = [run_step(ctx, cfg, w, B.Adam(), 1e-2) for _ in range(3)]
+        for r in runs[1:]:
+            for k in ("p", "theta_plus", "metagrad", "loss_plus", "loss_minus"):
+                assert np.array_equal(r[k], runs[0][k]), (cfg.name, k)
+            assert r["sumsq"] == runs[0]["sumsq"] and r["eps_fd"] == runs[0]["eps_fd"]
+
+
 def test_step_host_matches_step():
     cfg = W.CONFIGS["tiny"]
     w = W.mlp_workload(cfg, 0)
