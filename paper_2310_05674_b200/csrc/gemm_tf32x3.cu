@@ -521,15 +521,18 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     // N-tile: 16 for a narrow last layer; 64 when 128-wide tiles would leave SMs idle; else 128.
     // (Hidden layers never take 16: their tiles must also write the zero padding up to round_up32(N).)
     const int64_t tiles128 = (int64_t)((L.M + BM - 1) / BM) * ((L.N + 127) / 128) * 2;
-    // When even that leaves SMs idle the contraction is split over several CTAs per tile (split-K).
+    // Split-K (several CTAs per tile, partials added in split order by the last CTA to arrive) exists for
+    // contractions that are long relative to the grid, but measured slower than 64-wide tiles on every
+    // workload here (the partial-tile round trip costs more than the idle SMs), so it is off unless the
+    // SAMA_TC_SPLITS environment variable asks for it.
     const bool narrow_last = L.last && L.N <= 16;
-    int bn = narrow_last ? 16 : (L.N <= 64 ? 64 : 128);
+    int bn = narrow_last ? 16 : ((L.N <= 64 || tiles128 < ctx->sm_count) ? 64 : 128);
     if (ctx->tile_override == 64 || ctx->tile_override == 128) bn = ctx->tile_override;
     const int num_kb_total = Kp / BKF;
     int splits = 1;
     {
         const int64_t tiles = (int64_t)((L.M + BM - 1) / BM) * ((L.N + bn - 1) / bn) * 2;
-        int want = (int)(ctx->sm_count / (tiles > 0 ? tiles : 1));
+        int want = 1;
         if (const char* e = std::getenv("SAMA_TC_SPLITS")) want = std::atoi(e);
         if (want > 8) want = 8;
         const int by_k = num_kb_total / 4;  // at least 4 k-blocks per split
@@ -538,7 +541,6 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
         if (tiles > kTcCounters) want = 1;
         if (want > 1 && ctx->tc_ws && ctx->tc_counters) splits = want;
     }
-    (void)tiles128;
     CUtensorMap maps[4];
     const int a_slabs = L.shared_a ? 1 : 2;
     // a box never exceeds the tensor's extent; rows of the shared-memory tile that no copy fills only

@@ -286,6 +286,18 @@ def test_step_is_bitwise_reproducible(gemm_mode):
             assert r["sumsq"] == runs[0]["sumsq"] and r["eps_fd"] == runs[0]["eps_fd"]
 
 
+def test_split_k_option_matches_and_is_reproducible(monkeypatch):
+    """The optional split of the contraction over several CTAs per tile (SAMA_TC_SPLITS) adds its
+    partial tiles in a fixed order: same parity bar, bitwise repeatable."""
+    monkeypatch.setenv("SAMA_TC_SPLITS", "3")
+    cfg, w = W.custom_mlp((2048, 512, 300, 40), 200, seed=8)
+    check_step(cfg, w, B.Adam(), 1.0, gemm_mode=2)
+    with Ctx(cfg.n_params, cfg.batch, cfg.dims, 2) as ctx:
+        a = run_step(ctx, cfg, w, B.Adam(), 1.0)
+        b = run_step(ctx, cfg, w, B.Adam(), 1.0)
+    assert np.array_equal(a["metagrad"], b["metagrad"]) and np.array_equal(a["loss_plus"], b["loss_plus"])
+
+
 def test_step_host_matches_step():
     cfg = W.CONFIGS["tiny"]
     w = W.mlp_workload(cfg, 0)
