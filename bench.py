@@ -227,34 +227,26 @@ def main():
         return
 
     import torch
-    import torch.distributed as dist
     from paper_2310_05674_b200 import binding as S
+    from paper_2310_05674_b200 import replicas
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dev = "cuda:%d" % local
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+    group = replicas.init(backend="nccl", device=dev)   # one process per GPU; independent replicas
+    world, rank = group.world, group.rank
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        group.barrier()
         torch.cuda.synchronize()
 
     def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return group.max_over_ranks(x, dev)
 
     peaks = load_peaks()
     name = args.workload
     flat = name in W.FLAT_SIZES
-    seed = rank  # each rank owns an independent batch / vector: no data-path collective
+    seed = group.seed  # each rank owns an independent batch / vector: no data-path collective
     if flat:
         n = args.flat_n or W.FLAT_SIZES[name]
         w = W.flat_vector(n, seed)
@@ -421,8 +413,7 @@ def main():
     S.sama_destroy(ctx)
     if rank == 0:
         print(json.dumps(out), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    group.close()
 
 
 if __name__ == "__main__":

@@ -1,0 +1,68 @@
+"""Host-side plumbing for running independent replicas of the step, one process per GPU.
+
+The meta-gradient step does not shard in this library: each rank owns a whole
+problem (its own seeded batch and parameter vector) and there is no data-path
+collective.  What the ranks share is only measurement: a barrier on both sides
+of a timed region, the maximum of a duration over ranks, and the aggregate
+throughput (units processed by all ranks divided by that maximum).  The same
+code runs over NCCL on GPUs and over gloo on CPU (which is how it is tested).
+"""
+from __future__ import annotations
+
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+
+@dataclass
+class Replicas:
+    rank: int
+    world: int
+    local_rank: int
+    backend: Optional[str]  # None when world == 1
+
+    @property
+    def seed(self) -> int:
+        """Workload seed of this rank: every replica draws an independent problem."""
+        return self.rank
+
+    def barrier(self) -> None:
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+
+    def max_over_ranks(self, x: float, device: str = "cpu") -> float:
+        if self.world == 1:
+            return float(x)
+        import torch
+        import torch.distributed as dist
+        t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def aggregate_rate(self, units_per_rank: float, seconds_this_rank: float, device: str = "cpu") -> float:
+        """Whole-job throughput: all ranks' units over the slowest rank's time."""
+        return self.world * units_per_rank / self.max_over_ranks(seconds_this_rank, device)
+
+    def close(self) -> None:
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+def init(backend: str = "nccl", device: Optional[str] = None) -> Replicas:
+    """Reads RANK / LOCAL_RANK / WORLD_SIZE / MASTER_* from the environment and joins the group."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world == 1:
+        return Replicas(rank, world, local, None)
+    import torch
+    import torch.distributed as dist
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29500")
+    kw = {}
+    if backend == "nccl" and device is not None:
+        kw["device_id"] = torch.device(device)
+    dist.init_process_group(backend, rank=rank, world_size=world, **kw)
+    return Replicas(rank, world, local, backend)

@@ -1,0 +1,72 @@
+"""The N > 1 path of the benchmark on CPU: two gloo ranks as child processes.
+
+Ranks are independent replicas (no data-path collective); what they share is
+the timing protocol.  This checks the rank-dependent seeding, the barrier, the
+max-over-ranks reduction and the aggregate rate."""
+import os
+import socket
+import subprocess
+import sys
+import textwrap
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+CHILD = textwrap.dedent("""
+    import json, sys, time
+    sys.path.insert(0, %r)
+    import numpy as np
+    from paper_2310_05674_b200 import replicas, workloads as W
+    r = replicas.init(backend="gloo")
+    w = W.flat_vector(1000, r.seed)
+    r.barrier()
+    t = 0.5 + 0.25 * r.rank                     # pretend rank 1 is slower
+    out = {"rank": r.rank, "world": r.world, "seed": r.seed,
+           "theta0": float(w["theta"][0]),
+           "tmax": r.max_over_ranks(t),
+           "rate": r.aggregate_rate(10.0, t)}
+    r.barrier()
+    r.close()
+    print("RESULT " + json.dumps(out), flush=True)
+""") % ROOT
+
+
+def test_two_gloo_ranks_share_only_the_timing_protocol(tmp_path):
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    script = tmp_path / "child.py"
+    script.write_text(CHILD)
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE="2",
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env, stdout=subprocess.PIPE,
+                                      stderr=subprocess.PIPE, text=True))
+    import json
+    res = {}
+    for p in procs:
+        out, err = p.communicate(timeout=180)
+        assert p.returncode == 0, err[-2000:]
+        line = [l for l in out.splitlines() if l.startswith("RESULT ")][0]
+        d = json.loads(line[7:])
+        res[d["rank"]] = d
+    assert res[0]["world"] == res[1]["world"] == 2
+    assert (res[0]["seed"], res[1]["seed"]) == (0, 1)
+    assert res[0]["theta0"] != res[1]["theta0"]           # independent problems
+    assert res[0]["tmax"] == res[1]["tmax"] == 0.75        # slowest rank's time on every rank
+    assert abs(res[0]["rate"] - 2 * 10.0 / 0.75) < 1e-12   # all ranks' units over that time
+
+
+def test_single_process_needs_no_group():
+    sys.path.insert(0, ROOT)
+    from paper_2310_05674_b200 import replicas
+    env = {k: os.environ.pop(k) for k in ("WORLD_SIZE", "RANK", "LOCAL_RANK") if k in os.environ}
+    try:
+        r = replicas.init()
+        assert (r.rank, r.world, r.backend) == (0, 1, None)
+        assert r.max_over_ranks(1.5) == 1.5 and r.aggregate_rate(3.0, 1.5) == 2.0
+        r.barrier()
+        r.close()
+    finally:
+        os.environ.update(env)
