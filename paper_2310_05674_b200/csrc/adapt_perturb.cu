@@ -292,6 +292,8 @@ __global__ void __launch_bounds__(kThreads)
 perturb_split_kernel(int64_t n, const float* theta, const float* __restrict__ p, const double* __restrict__ sumsq,
                      float alpha, float* theta_plus, float* theta_minus, DeviceScalars* sc, float* eps_fd_out,
                      SplitLayout lay, float* __restrict__ hi, float* __restrict__ lo) {
+    pdl_trigger();
+    pdl_wait();  // p and the sum of squares come from the adaptation kernel just before
     bool bad;
     const float eps = step_size(*sumsq, alpha, bad);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -431,9 +433,8 @@ cudaError_t launch_perturb_split(sama_ctx* ctx, int64_t n, const float* theta, c
                                  float alpha, float* theta_plus, float* theta_minus, float* eps_fd_out,
                                  const SplitLayout& lay, float* hi, float* lo, cudaStream_t st) {
     KernelScope scope(ctx, SAMA_K_PERTURB_SPLIT, -1, st);
-    perturb_split_kernel<<<stream_grid(ctx, n >> 2, kUnroll), kThreads, 0, st>>>(
-        n, theta, p, sumsq, alpha, theta_plus, theta_minus, ctx->scalars, eps_fd_out, lay, hi, lo);
-    return cudaGetLastError();
+    return launch_dependent(perturb_split_kernel, dim3(stream_grid(ctx, n >> 2, kUnroll)), dim3(kThreads), 0, st, n,
+                            theta, p, sumsq, alpha, theta_plus, theta_minus, ctx->scalars, eps_fd_out, lay, hi, lo);
 }
 
 }  // namespace sama

@@ -39,6 +39,8 @@ ce_fd_kernel(const float* __restrict__ zp, const float* __restrict__ zm, int ldz
              const float* __restrict__ lambda, int B, int C, const float* __restrict__ eps_fd,
              float* __restrict__ metagrad, float* __restrict__ loss_plus, float* __restrict__ loss_minus,
              DeviceScalars* sc) {
+    pdl_trigger();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int i = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     if (i >= B) return;
@@ -70,9 +72,8 @@ cudaError_t launch_ce_fd(sama_ctx* ctx, const float* z_plus, const float* z_minu
                          float* loss_plus, float* loss_minus, cudaStream_t st) {
     const int grid = (B + kWarpsPerBlock - 1) / kWarpsPerBlock;
     KernelScope scope(ctx, SAMA_K_CE_FD, -1, st);
-    ce_fd_kernel<<<grid, kWarpsPerBlock * 32, 0, st>>>(z_plus, z_minus, ldz, y, lambda, B, C, eps_fd, metagrad,
-                                                       loss_plus, loss_minus, ctx->scalars);
-    return cudaGetLastError();
+    return launch_dependent(ce_fd_kernel, dim3(grid), dim3(kWarpsPerBlock * 32), 0, st, z_plus, z_minus, ldz, y, lambda,
+                            B, C, eps_fd, metagrad, loss_plus, loss_minus, ctx->scalars);
 }
 
 }  // namespace sama

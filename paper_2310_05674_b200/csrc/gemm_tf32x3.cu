@@ -215,6 +215,10 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr_slot;
+    // everything above (barriers, tensor memory) overlapped the previous kernel's tail; its outputs
+    // (our operands) are only touched from here on
+    pdl_trigger();
+    pdl_wait();
 
     auto raise_timeout = [&]() {
         *abort_flag = 1;
@@ -404,6 +408,8 @@ struct SplitArgs {
 template <bool VEC>
 __global__ void __launch_bounds__(256)
 split_tf32_kernel(SplitArgs a) {
+    pdl_trigger();
+    pdl_wait();
     const int br = blockIdx.z;
     const float* __restrict__ src = br ? a.src[1] : a.src[0];
     float* __restrict__ hi = a.hi + (int64_t)br * a.slab;
@@ -479,8 +485,8 @@ cudaError_t launch_tc(const CUtensorMap maps[4], const TcArgs& a, dim3 grid, cud
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    gemm_tf32x3_kernel<BN><<<grid, kThreads, smem_bytes(BN), st>>>(maps[0], maps[1], maps[2], maps[3], a);
-    return cudaGetLastError();
+    return launch_dependent(gemm_tf32x3_kernel<BN>, grid, dim3(kThreads), (size_t)smem_bytes(BN), st, maps[0], maps[1],
+                            maps[2], maps[3], a);
 }
 
 inline int round_up32(int x) { return (x + 31) & ~31; }
@@ -506,11 +512,9 @@ cudaError_t launch_split_tf32(sama_ctx* ctx, const float* src0, const float* src
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     KernelScope scope(ctx, SAMA_K_SPLIT, -1, st);
-    if (vec)
-        split_tf32_kernel<true><<<dim3((unsigned)blocks, 1, branches), 256, 0, st>>>(a);
-    else
-        split_tf32_kernel<false><<<dim3((unsigned)blocks, 1, branches), 256, 0, st>>>(a);
-    return cudaGetLastError();
+    const dim3 grid((unsigned)blocks, 1, branches);
+    return vec ? launch_dependent(split_tf32_kernel<true>, grid, dim3(256), 0, st, a)
+               : launch_dependent(split_tf32_kernel<false>, grid, dim3(256), 0, st, a);
 }
 
 // One layer on the tensor cores.  a_hi/a_lo: [shared_a ? 1 : 2][M][Kp]; w_hi/w_lo: [2][N][Kp]; Kp = K rounded

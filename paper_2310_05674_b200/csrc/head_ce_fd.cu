@@ -28,6 +28,8 @@ head_ce_fd_kernel(const float* __restrict__ hp, const float* __restrict__ hm, in
                   const int32_t* __restrict__ y, const float* __restrict__ lambda, int B, int C, int K,
                   const float* __restrict__ eps_fd, float* __restrict__ metagrad,
                   float* __restrict__ loss_plus, float* __restrict__ loss_minus, DeviceScalars* sc) {
+    pdl_trigger();
+    pdl_wait();
     constexpr int SPB = kWarps / WPS;  // samples per block
     __shared__ float part[kWarps][2 * CT];
     __shared__ float tot[SPB][2 * CT];
@@ -144,17 +146,18 @@ cudaError_t launch_head_ce_fd(sama_ctx* ctx, const float* h_plus, const float* h
     const bool wide = (int64_t)B <= 8 * (int64_t)ctx->sm_count;
     const int grid = wide ? B : (B + kWarps - 1) / kWarps;
     KernelScope scope(ctx, SAMA_K_HEAD, -1, st);
+    cudaError_t err = cudaSuccess;
 #define SAMA_HEAD2(CT, V, W)                                                                                       \
-    head_ce_fd_kernel<CT, V, W><<<grid, kWarps * 32, 0, st>>>(h_plus, h_minus, ldh, w_plus, w_minus, b_plus,       \
-                                                              b_minus, y, lambda, B, C, K, eps_fd, metagrad,       \
-                                                              loss_plus, loss_minus, ctx->scalars)
+    err = launch_dependent(head_ce_fd_kernel<CT, V, W>, dim3(grid), dim3(kWarps * 32), 0, st, h_plus, h_minus, ldh, \
+                           w_plus, w_minus, b_plus, b_minus, y, lambda, B, C, K, eps_fd, metagrad, loss_plus,      \
+                           loss_minus, ctx->scalars)
 #define SAMA_HEAD(CT, V) do { if (wide) SAMA_HEAD2(CT, V, 8); else SAMA_HEAD2(CT, V, 1); } while (0)
     if (C <= 4) { if (vec) SAMA_HEAD(4, true); else SAMA_HEAD(4, false); }
     else if (C <= 10) { if (vec) SAMA_HEAD(10, true); else SAMA_HEAD(10, false); }
     else { if (vec) SAMA_HEAD(16, true); else SAMA_HEAD(16, false); }
 #undef SAMA_HEAD
 #undef SAMA_HEAD2
-    return cudaGetLastError();
+    return err;
 }
 
 }  // namespace sama

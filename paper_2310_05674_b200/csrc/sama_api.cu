@@ -307,6 +307,10 @@ int run_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const 
 }  // namespace
 
 namespace sama {
+bool pdl_enabled() {
+    static const bool on = []() { const char* e = std::getenv("SAMA_NO_PDL"); return !(e && e[0] == '1'); }();
+    return on;
+}
 cudaError_t launch_gemm(sama_ctx* ctx, const GemmArgs& g, cudaStream_t st) {
     return launch_gemm_ffma(ctx, g, st);
 }

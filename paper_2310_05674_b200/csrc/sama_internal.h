@@ -112,6 +112,30 @@ int check_adam(const sama_adam_t* a, AdaptConsts* out);
 int validate_adapt(int64_t max_n, int64_t n, const float* m, const float* s, const float* g_base,
                    const float* g_meta, const sama_adam_t* adam, float* p_out, double* sumsq_out, AdaptConsts* c);
 
+// Programmatic dependent launch: a kernel launched this way may start (and run its prologue) while
+// the previous kernel on the stream is still finishing; it must execute pdl_wait() before it touches
+// anything the previous kernels wrote or still read.  pdl_wait() is a no-op under a plain launch.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+bool pdl_enabled();
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                             Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // adapt_perturb.cu
 cudaError_t launch_adapt_sumsq(sama_ctx* ctx, int64_t n, const float* m, const float* s, const float* g_base,
                                const float* g_meta, const AdaptConsts& c, float* p_out, double* sumsq_out,
