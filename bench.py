@@ -343,7 +343,8 @@ def main():
     if "perturb" in per_kernel:
         rooflines["perturb"] = hbm_roof("perturb", 16.0 * n)
     if "perturb_split" in per_kernel:  # perturb + TF32 hi/lo of both branches: 8 read + 8 + 16 written per element
-        rooflines["perturb_split"] = hbm_roof("perturb_split", 32.0 * n)
+        # ... plus the batch's operand split done by the same sweep: 4 read + 8 written per element of X
+        rooflines["perturb_split"] = hbm_roof("perturb_split", 32.0 * n + (12.0 * B * cfg.dims[0] if cfg else 0.0))
     for gk in ("gemm_ffma", "gemm_tf32x3"):
         if gk in per_kernel and cfg:
             flops = float(cfg.forward_flops)

@@ -291,8 +291,23 @@ __device__ __forceinline__ void tf32_split(float4 x, float4& h, float4& l) {
 __global__ void __launch_bounds__(kThreads)
 perturb_split_kernel(int64_t n, const float* theta, const float* __restrict__ p, const double* __restrict__ sumsq,
                      float alpha, float* theta_plus, float* theta_minus, DeviceScalars* sc, float* eps_fd_out,
-                     SplitLayout lay, float* __restrict__ hi, float* __restrict__ lo) {
+                     SplitLayout lay, float* __restrict__ hi, float* __restrict__ lo, XSplitJob xjob) {
     pdl_trigger();
+    // The batch does not depend on the adaptation: its operand split runs before the wait, i.e. while
+    // the previous kernel may still be draining.
+    if (xjob.rows > 0) {
+        const int q = xjob.ld_out >> 2;
+        const int64_t total = xjob.rows * q, xstride = (int64_t)gridDim.x * kThreads;
+        for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < total; i += xstride) {
+            const int64_t r = i / q;
+            const int c = (int)(i - r * q) << 2;
+            float4 x = make_float4(0.f, 0.f, 0.f, 0.f), h, l;
+            if (c < xjob.cols) x = __ldg(reinterpret_cast<const float4*>(xjob.x + r * xjob.cols + c));
+            tf32_split(x, h, l);
+            *reinterpret_cast<float4*>(xjob.hi + r * xjob.ld_out + c) = h;
+            *reinterpret_cast<float4*>(xjob.lo + r * xjob.ld_out + c) = l;
+        }
+    }
     pdl_wait();  // p and the sum of squares come from the adaptation kernel just before
     bool bad;
     const float eps = step_size(*sumsq, alpha, bad);
@@ -431,10 +446,10 @@ bool perturb_split_applicable(const SplitLayout& lay, const float* theta, const 
 
 cudaError_t launch_perturb_split(sama_ctx* ctx, int64_t n, const float* theta, const float* p, const double* sumsq,
                                  float alpha, float* theta_plus, float* theta_minus, float* eps_fd_out,
-                                 const SplitLayout& lay, float* hi, float* lo, cudaStream_t st) {
+                                 const SplitLayout& lay, float* hi, float* lo, const XSplitJob& xjob, cudaStream_t st) {
     KernelScope scope(ctx, SAMA_K_PERTURB_SPLIT, -1, st);
     return launch_dependent(perturb_split_kernel, dim3(stream_grid(ctx, n >> 2, kUnroll)), dim3(kThreads), 0, st, n,
-                            theta, p, sumsq, alpha, theta_plus, theta_minus, ctx->scalars, eps_fd_out, lay, hi, lo);
+                            theta, p, sumsq, alpha, theta_plus, theta_minus, ctx->scalars, eps_fd_out, lay, hi, lo, xjob);
 }
 
 }  // namespace sama

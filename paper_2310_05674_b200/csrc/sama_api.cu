@@ -184,11 +184,16 @@ bool tc_fits(const sama_ctx* ctx, const sama_mlp_t* mlp, int32_t B) {
     return true;
 }
 
+// A single-layer model with a narrow output runs entirely in the fused head: no tensor-core product, no X split.
+bool fused_head_only_model(const sama_mlp_t* mlp) {
+    return mlp->n_layers == 1 && head_applicable(mlp->dims[1]);
+}
+
 // Forward pass of both branches on the tensor cores (3xTF32).  Operands are TF32 hi/lo pairs: X is split
 // here, hidden activations by the epilogue that produces them, and the weights either by the fused
 // perturbation sweep (w_presplit) or here, layer by layer.
 int run_forward_tc(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const float* theta_minus,
-                   const float* X, int32_t B, bool w_presplit, bool fused_head, cudaStream_t st) {
+                   const float* X, int32_t B, bool w_presplit, bool x_presplit, bool fused_head, cudaStream_t st) {
     // with a fused head the last layer is not a matrix product here, and the layer before it
     // leaves fp32 activations (ReLU applied) in the context's activation buffer
     const int L = fused_head ? mlp->n_layers - 1 : mlp->n_layers;
@@ -197,8 +202,9 @@ int run_forward_tc(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus
     const SplitLayout lay = make_split_layout(mlp);
     float* w_hi = ctx->w_split;
     float* w_lo = ctx->w_split + ctx->w_split_half;
-    SAMA_CUDA(ctx, launch_split_tf32(ctx, X, X, 1, B, mlp->dims[0], ctx->x_split, ctx->x_split + ctx->x_split_half,
-                                     0, st));
+    if (!x_presplit)
+        SAMA_CUDA(ctx, launch_split_tf32(ctx, X, X, 1, B, mlp->dims[0], ctx->x_split,
+                                         ctx->x_split + ctx->x_split_half, 0, st));
     for (int l = 0; l < L; ++l) {
         const int din = mlp->dims[l], dout = mlp->dims[l + 1];
         const bool last = (l + 1 == L);
@@ -239,7 +245,7 @@ int run_forward_tc(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus
 int run_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const float* theta_minus,
            const float* X, const int32_t* y, const float* lambda, int32_t B, const float* eps_fd,
            float* metagrad_out, float* loss_plus_out, float* loss_minus_out, cudaStream_t st,
-           bool w_presplit = false) {
+           bool w_presplit = false, bool x_presplit = false) {
     const int L = mlp->n_layers;
     const int C = mlp->dims[L];
     const bool fits = tc_fits(ctx, mlp, B);
@@ -252,7 +258,7 @@ int run_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const 
     int ld_in = mlp->dims[0];
 
     if (use_tc) {
-        const int rc = run_forward_tc(ctx, mlp, theta_plus, theta_minus, X, B, w_presplit, fused_head, st);
+        const int rc = run_forward_tc(ctx, mlp, theta_plus, theta_minus, X, B, w_presplit, x_presplit, fused_head, st);
         if (rc != SAMA_OK) return rc;
         if (n_gemm > 0) {
             float* out = fused_head ? ctx->act[0] : ctx->logits;
@@ -499,15 +505,28 @@ int sama_step(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* thet
     const SplitLayout lay = make_split_layout(mlp);
     const bool fused = ctx->gemm_mode != 1 && tc_fits(ctx, mlp, B) &&
                        perturb_split_applicable(lay, theta, p_out, theta_plus, theta_minus);
+    // ... and, where the batch allows vector access, the split of X as well (one launch fewer)
+    XSplitJob xjob;
+    std::memset(&xjob, 0, sizeof(xjob));
+    const bool x_fused = fused && (mlp->dims[0] % 4 == 0) && aligned(X, 16) &&
+                         !(fused_head_only_model(mlp));
+    if (x_fused) {
+        xjob.x = X;
+        xjob.hi = ctx->x_split;
+        xjob.lo = ctx->x_split + ctx->x_split_half;
+        xjob.rows = B;
+        xjob.cols = mlp->dims[0];
+        xjob.ld_out = (mlp->dims[0] + 31) & ~31;
+    }
     if (fused)
         SAMA_CUDA(ctx, launch_perturb_split(ctx, n, theta, p_out, &ctx->scalars->sumsq, alpha, theta_plus,
                                             theta_minus, nullptr, lay, ctx->w_split,
-                                            ctx->w_split + ctx->w_split_half, st));
+                                            ctx->w_split + ctx->w_split_half, xjob, st));
     else
         SAMA_CUDA(ctx, launch_perturb(ctx, n, theta, p_out, &ctx->scalars->sumsq, alpha, theta_plus, theta_minus,
                                       nullptr, st));
     return run_fd(ctx, mlp, theta_plus, theta_minus, X, y, lambda, B, nullptr, metagrad_out, loss_plus_out,
-                  loss_minus_out, st, fused);
+                  loss_minus_out, st, fused, x_fused);
 }
 
 int sama_step_host(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* theta_host, const float* m_host,

@@ -45,6 +45,16 @@ struct SplitLayout {
     int64_t slab;               // floats per slab = sum_l d_l * Kp_l
 };
 
+// The batch X as an extra job of the fused perturbation sweep: its TF32 hi/lo split, rows padded to ld_out.
+// rows == 0 means "no X job".  Requires cols % 4 == 0 and a 16-byte aligned X.
+struct XSplitJob {
+    const float* x;
+    float* hi;
+    float* lo;
+    int64_t rows;
+    int cols, ld_out;
+};
+
 struct ProfRecord {
     int kind, layer;
     cudaEvent_t start, stop;
@@ -148,7 +158,7 @@ bool perturb_split_applicable(const SplitLayout& lay, const float* theta, const 
                               const float* theta_minus);
 cudaError_t launch_perturb_split(sama_ctx* ctx, int64_t n, const float* theta, const float* p, const double* sumsq,
                                  float alpha, float* theta_plus, float* theta_minus, float* eps_fd_out,
-                                 const SplitLayout& lay, float* hi, float* lo, cudaStream_t st);
+                                 const SplitLayout& lay, float* hi, float* lo, const XSplitJob& xjob, cudaStream_t st);
 
 // One layer of both branches: C[b] = act(A[b] * W[b]^T + bias[b]) for b in {0, 1}
 struct GemmArgs {
