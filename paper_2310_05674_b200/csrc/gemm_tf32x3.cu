@@ -42,9 +42,12 @@ constexpr int UMMA_K = 8;     // K of one kind::tf32 instruction
 constexpr int kThreads = 192;
 constexpr long long kWaitCycles = 4000000000LL;  // ~2 s at 2 GHz
 
-__host__ __device__ constexpr int stages_for(int bn) { return bn >= 128 ? 3 : 4; }
-__host__ __device__ constexpr int stage_bytes(int bn) { return 2 * BM * BKF * 4 + 2 * bn * BKF * 4; }
-__host__ __device__ constexpr int smem_bytes(int bn) { return stages_for(bn) * stage_bytes(bn) + 1024 + 256; }
+// `wrows` = rows of W one CTA stages per k-block: BN, or BN / 2 when a CTA pair shares the W tile.
+__host__ __device__ constexpr int stage_bytes(int wrows) { return 2 * BM * BKF * 4 + 2 * wrows * BKF * 4; }
+__host__ __device__ constexpr int stages_for(int wrows) {
+    return (200 * 1024) / stage_bytes(wrows) > 5 ? 5 : (200 * 1024) / stage_bytes(wrows);
+}
+__host__ __device__ constexpr int smem_bytes(int wrows) { return stages_for(wrows) * stage_bytes(wrows) + 1024 + 256; }
 
 // ---------------------------------------------------------------- PTX wrappers
 
@@ -81,6 +84,48 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
+}
+
+// CTA-pair (cta_group::2) forms.  Shared-memory addresses of a cluster carry the CTA rank in bit 24:
+// clearing it names the same offset in the even ("leader") CTA of the pair.
+constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu;
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Load into THIS CTA's shared memory; completion bytes are signalled on the leader's mbarrier.  No multicast.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t leader_bar, int x, int y, int z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(leader_bar), "r"(x), "r"(y), "r"(z) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t slot, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// One instruction drives both SMs: D (256 x N, 128 rows in each CTA's tensor memory) += A (each CTA's 128 rows)
+// x B^T (N rows, half of them staged by each CTA).
+__device__ __forceinline__ void umma_tf32_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrives on the barrier at this offset in both CTAs of the pair once the products issued so far are done.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    asm volatile(
+        "{\n\t.reg .b16 m;\n\tmov.b16 m, 3;\n\t"
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n\t}"
+        ::"r"(bar) : "memory");
 }
 
 __device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols) {
@@ -129,8 +174,8 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
 
 // Instruction descriptor: D = fp32 (1 at bit 4), A and B = TF32 (2 at bits 7 and
 // 10), both K-major (bits 15, 16 clear), N/8 at bit 17, M/16 at bit 24.
-__host__ __device__ constexpr uint32_t make_idesc(int n) {
-    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+__host__ __device__ constexpr uint32_t make_idesc(int n, int m = BM) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 __device__ __forceinline__ float to_tf32(float x) {
@@ -155,16 +200,20 @@ struct TcArgs {
     int32_t* status;
 };
 
-template <int BN>
+// PAIR = true: two CTAs of a cluster work on one 256 x BN tile.  Each stages its own 128 rows of A and half of
+// the W tile; the leader CTA issues cta_group::2 products that read both CTAs' shared memory and write both
+// CTAs' tensor memory.  Per CTA and flop that is fewer operand bytes than two independent 128 x BN tiles.
+template <int BN, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
                    const __grid_constant__ CUtensorMap map_w_hi, const __grid_constant__ CUtensorMap map_w_lo,
                    TcArgs args) {
-    constexpr int STAGES = stages_for(BN);
-    constexpr int A_BYTES = BM * BKF * 4, W_BYTES = BN * BKF * 4;
-    constexpr int STAGE = stage_bytes(BN);
+    constexpr int WROWS = PAIR ? BN / 2 : BN;  // rows of W this CTA stages
+    constexpr int STAGES = stages_for(WROWS);
+    constexpr int A_BYTES = BM * BKF * 4, W_BYTES = WROWS * BKF * 4;
+    constexpr int STAGE = stage_bytes(WROWS);
     constexpr uint32_t TMEM_COLS = BN < 32 ? 32 : BN;
-    constexpr uint32_t IDESC = make_idesc(BN);
+    constexpr uint32_t IDESC = make_idesc(BN, PAIR ? 2 * BM : BM);
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // tiles need 1024-byte alignment
@@ -185,18 +234,21 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int br = blockIdx.z / args.splits, split = blockIdx.z - br * args.splits;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;  // 0 = leader of the pair
+    const int tile_id = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     // Tile order: CTAs that run together cover all M-tiles of a group of `group_n` N-tiles, so one wave
     // re-uses a bounded set of W tiles and every A tile from L2 instead of sweeping all of W.
     int tile_m, tile_n;
     {
         const int per_group = args.group_n * args.tiles_m;
-        const int group = blockIdx.x / per_group, rem = blockIdx.x - group * per_group;
+        const int group = tile_id / per_group, rem = tile_id - group * per_group;
         const int first_n = group * args.group_n;
         const int gsz = min(args.group_n, args.tiles_n - first_n);
         tile_n = first_n + rem % gsz;
         tile_m = rem / gsz;
     }
-    const int m0 = tile_m * BM, n0 = tile_n * BN;
+    const int m0 = tile_m * (PAIR ? 2 * BM : BM) + (int)rank * BM, n0 = tile_n * BN;
+    const int nw0 = n0 + (int)rank * WROWS;  // first W row this CTA stages
     // this CTA's share of the contraction (the host guarantees at least one k-block per split)
     const int kb_begin = split * args.kb_per_split;
     const int num_kb = min(args.kb_per_split, args.num_kb - kb_begin);
@@ -210,9 +262,12 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);
+    if (warp == 1) {
+        if (PAIR) tmem_alloc_pair(tmem_slot, TMEM_COLS); else tmem_alloc(tmem_slot, TMEM_COLS);
+    }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync();  // the peer's barriers exist before anything is signalled on them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr_slot;
     // everything above (barriers, tensor memory) overlapped the previous kernel's tail; its outputs
@@ -236,23 +291,33 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                 if (kb >= STAGES && !mbar_wait(empty_bar(s), (round - 1) & 1)) { raise_timeout(); break; }
                 if (*abort_flag) break;
                 const uint32_t st = base + s * STAGE;
-                mbar_expect_tx(full_bar(s), args.tx_bytes);
                 const int kx = (kb_begin + kb) * BKF;
-                tma_load_3d(st, &map_a_hi, full_bar(s), kx, m0, za);
-                tma_load_3d(st + A_BYTES, &map_a_lo, full_bar(s), kx, m0, za);
-                tma_load_3d(st + 2 * A_BYTES, &map_w_hi, full_bar(s), kx, n0, br);
-                tma_load_3d(st + 2 * A_BYTES + W_BYTES, &map_w_lo, full_bar(s), kx, n0, br);
+                if (PAIR) {
+                    // both CTAs' copies complete on the leader's barrier, which the leader arms for all of them
+                    const uint32_t lbar = full_bar(s) & kPeerBitMask;
+                    if (rank == 0) mbar_expect_tx(full_bar(s), args.tx_bytes);
+                    tma_load_3d_pair(st, &map_a_hi, lbar, kx, m0, za);
+                    tma_load_3d_pair(st + A_BYTES, &map_a_lo, lbar, kx, m0, za);
+                    tma_load_3d_pair(st + 2 * A_BYTES, &map_w_hi, lbar, kx, nw0, br);
+                    tma_load_3d_pair(st + 2 * A_BYTES + W_BYTES, &map_w_lo, lbar, kx, nw0, br);
+                } else {
+                    mbar_expect_tx(full_bar(s), args.tx_bytes);
+                    tma_load_3d(st, &map_a_hi, full_bar(s), kx, m0, za);
+                    tma_load_3d(st + A_BYTES, &map_a_lo, full_bar(s), kx, m0, za);
+                    tma_load_3d(st + 2 * A_BYTES, &map_w_hi, full_bar(s), kx, n0, br);
+                    tma_load_3d(st + 2 * A_BYTES + W_BYTES, &map_w_lo, full_bar(s), kx, n0, br);
+                }
                 issued = kb + 1;
             }
-            if (*abort_flag) {
+            if (*abort_flag && rank == 0) {
                 // let the copies already issued land before the CTA's shared memory goes away
                 for (int kb = (issued > STAGES ? issued - STAGES : 0); kb < issued; ++kb)
                     mbar_wait(full_bar(kb % STAGES), (kb / STAGES) & 1);
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------ MMA issuer (the leader's, for a pair)
+        if (lane == 0 && rank == 0) {
             bool ok = true;
             for (int kb = 0; kb < num_kb && ok; ++kb) {
                 const int s = kb % STAGES;
@@ -265,13 +330,20 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
 #pragma unroll
                 for (int k = 0; k < BKF / UMMA_K; ++k) {
                     const uint64_t adv = (uint64_t)((k * UMMA_K * 4) >> 4);  // 32 bytes per k-step inside the swizzled row
-                    umma_tf32(tmem_base, a_hi + adv, w_lo + adv, IDESC, (kb | k) != 0);
-                    umma_tf32(tmem_base, a_lo + adv, w_hi + adv, IDESC, 1);
-                    umma_tf32(tmem_base, a_hi + adv, w_hi + adv, IDESC, 1);
+                    if (PAIR) {
+                        umma_tf32_pair(tmem_base, a_hi + adv, w_lo + adv, IDESC, (kb | k) != 0);
+                        umma_tf32_pair(tmem_base, a_lo + adv, w_hi + adv, IDESC, 1);
+                        umma_tf32_pair(tmem_base, a_hi + adv, w_hi + adv, IDESC, 1);
+                    } else {
+                        umma_tf32(tmem_base, a_hi + adv, w_lo + adv, IDESC, (kb | k) != 0);
+                        umma_tf32(tmem_base, a_lo + adv, w_hi + adv, IDESC, 1);
+                        umma_tf32(tmem_base, a_hi + adv, w_hi + adv, IDESC, 1);
+                    }
                 }
-                umma_commit(empty_bar(s));  // frees the stage once these products have read it
+                // frees the stage (in both CTAs of a pair) once these products have read it
+                if (PAIR) umma_commit_pair(empty_bar(s)); else umma_commit(empty_bar(s));
             }
-            if (ok) umma_commit(accum_bar);
+            if (ok) { if (PAIR) umma_commit_pair(accum_bar); else umma_commit(accum_bar); }
         }
     } else {
         // -------------------------------------------------------------- epilogue
@@ -388,9 +460,10 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync();  // neither CTA leaves (or frees tensor memory) while the other may still use it
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, TMEM_COLS);
+        if (PAIR) tmem_dealloc_pair(tmem_base, TMEM_COLS); else tmem_dealloc(tmem_base, TMEM_COLS);
     }
 }
 
@@ -476,17 +549,18 @@ bool make_map(CUtensorMap* map, const float* base, int ld, int64_t rows, int sla
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN>
+template <int BN, bool PAIR>
 cudaError_t launch_tc(const CUtensorMap maps[4], const TcArgs& a, dim3 grid, cudaStream_t st) {
+    constexpr int kSmem = smem_bytes(PAIR ? BN / 2 : BN);
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tf32x3_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             smem_bytes(BN));
+        cudaError_t e = cudaFuncSetAttribute(gemm_tf32x3_kernel<BN, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kSmem);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    return launch_dependent(gemm_tf32x3_kernel<BN>, grid, dim3(kThreads), (size_t)smem_bytes(BN), st, maps[0], maps[1],
-                            maps[2], maps[3], a);
+    return launch_clustered(PAIR ? 2 : 1, gemm_tf32x3_kernel<BN, PAIR>, grid, dim3(kThreads), (size_t)kSmem, st,
+                            maps[0], maps[1], maps[2], maps[3], a);
 }
 
 inline int round_up32(int x) { return (x + 31) & ~31; }
@@ -545,11 +619,22 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
         if (tiles > kTcCounters) want = 1;
         if (want > 1 && ctx->tc_ws && ctx->tc_counters) splits = want;
     }
+    // CTA pairs (256 x bn tiles) when the batch spans at least two 128-row tiles: per CTA and flop they stage
+    // fewer operand bytes, which is what bounds this kernel.  bn = 128 while that still fills the machine.
+    bool pair = !narrow_last && splits == 1 && L.M > BM && L.N >= 64;
+    if (const char* e = std::getenv("SAMA_TC_PAIR")) pair = pair && std::atoi(e) != 0;
+    if (pair) {
+        const int64_t pairs128 = (int64_t)((L.M + 2 * BM - 1) / (2 * BM)) * ((L.N + 127) / 128) * 2;
+        bn = (L.N >= 128 && 2 * pairs128 >= ctx->sm_count) ? 128 : 64;
+        if (ctx->tile_override == 64 || ctx->tile_override == 128 || ctx->tile_override == 256) bn = ctx->tile_override;
+        if (L.N < bn) pair = false;
+    }
     CUtensorMap maps[4];
     const int a_slabs = L.shared_a ? 1 : 2;
     // a box never exceeds the tensor's extent; rows of the shared-memory tile that no copy fills only
     // feed output rows / columns that the epilogue does not store
-    const int a_box = L.M < BM ? L.M : BM, w_box = L.N < bn ? L.N : bn;
+    const int wrows = pair ? bn / 2 : bn;
+    const int a_box = L.M < BM ? L.M : BM, w_box = L.N < wrows ? L.N : wrows;
     const int64_t a_slab = (int64_t)L.M * Kp;
     if (!make_map(&maps[0], L.a_hi, Kp, L.M, a_slabs, a_box, a_slab) ||
         !make_map(&maps[1], L.a_lo, Kp, L.M, a_slabs, a_box, a_slab) ||
@@ -570,9 +655,9 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     a.relu = L.relu;
     a.last = L.last;
     a.shared_a = L.shared_a;
-    a.tx_bytes = (uint32_t)(2 * a_box * BKF * 4 + 2 * w_box * BKF * 4);
+    a.tx_bytes = (uint32_t)(2 * a_box * BKF * 4 + 2 * w_box * BKF * 4) * (pair ? 2u : 1u);  // a pair's barrier counts both CTAs' copies
     a.status = &ctx->scalars->status;
-    a.tiles_m = (L.M + BM - 1) / BM;
+    a.tiles_m = pair ? (L.M + 2 * BM - 1) / (2 * BM) : (L.M + BM - 1) / BM;
     a.tiles_n = (L.N + bn - 1) / bn;
     // about one wave of CTAs per group: group_n N-tiles x all M-tiles
     a.kb_per_split = (num_kb_total + splits - 1) / splits;
@@ -583,11 +668,16 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     if (a.group_n < 1) a.group_n = 1;
     if (a.group_n > a.tiles_n) a.group_n = a.tiles_n;
     if (const char* e = std::getenv("SAMA_TC_GROUP")) { const int g = std::atoi(e); if (g >= 1 && g <= a.tiles_n) a.group_n = g; }
-    dim3 grid(a.tiles_m * a.tiles_n, 1, 2 * a.splits);
+    dim3 grid(a.tiles_m * a.tiles_n * (pair ? 2 : 1), 1, 2 * a.splits);
     KernelScope scope(ctx, SAMA_K_GEMM_TF32X3, L.layer, st);
-    if (bn == 16) return launch_tc<16>(maps, a, grid, st);
-    if (bn == 64) return launch_tc<64>(maps, a, grid, st);
-    return launch_tc<128>(maps, a, grid, st);
+    if (pair) {
+        if (bn == 64) return launch_tc<64, true>(maps, a, grid, st);
+        if (bn == 256) return launch_tc<256, true>(maps, a, grid, st);
+        return launch_tc<128, true>(maps, a, grid, st);
+    }
+    if (bn == 16) return launch_tc<16, false>(maps, a, grid, st);
+    if (bn == 64) return launch_tc<64, false>(maps, a, grid, st);
+    return launch_tc<128, false>(maps, a, grid, st);
 }
 
 }  // namespace sama
