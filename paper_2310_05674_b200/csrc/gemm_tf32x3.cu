@@ -619,15 +619,18 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
         if (tiles > kTcCounters) want = 1;
         if (want > 1 && ctx->tc_ws && ctx->tc_counters) splits = want;
     }
-    // CTA pairs (256 x bn tiles) when the batch spans at least two 128-row tiles: per CTA and flop they stage
-    // fewer operand bytes, which is what bounds this kernel.  bn = 128 while that still fills the machine.
-    bool pair = !narrow_last && splits == 1 && L.M > BM && L.N >= 64;
+    // CTA pairs (256 x bn tiles): per CTA and flop they stage fewer operand bytes, which is what bounds this
+    // kernel -- but only worth it when the pairs still fill the machine (measured: wide4096 and head1024 gain
+    // 10 %, mlp3072 loses 4 %).  The widest pair tile whose grid covers every SM is taken.
+    bool pair = !narrow_last && splits == 1 && L.M > BM && L.N >= 128;
     if (const char* e = std::getenv("SAMA_TC_PAIR")) pair = pair && std::atoi(e) != 0;
     if (pair) {
-        const int64_t pairs128 = (int64_t)((L.M + 2 * BM - 1) / (2 * BM)) * ((L.N + 127) / 128) * 2;
-        bn = (L.N >= 128 && 2 * pairs128 >= ctx->sm_count) ? 128 : 64;
-        if (ctx->tile_override == 64 || ctx->tile_override == 128 || ctx->tile_override == 256) bn = ctx->tile_override;
-        if (L.N < bn) pair = false;
+        auto ctas = [&](int w) { return 2 * (int64_t)((L.M + 2 * BM - 1) / (2 * BM)) * ((L.N + w - 1) / w) * 2; };
+        int pbn = 0;
+        if (L.N >= 256 && ctas(256) >= ctx->sm_count) pbn = 256;
+        else if (ctas(128) >= ctx->sm_count) pbn = 128;
+        if (ctx->tile_override == 64 || ctx->tile_override == 128 || ctx->tile_override == 256) pbn = ctx->tile_override;
+        if (pbn == 0 || L.N < pbn) pair = false; else bn = pbn;
     }
     CUtensorMap maps[4];
     const int a_slabs = L.shared_a ? 1 : 2;
