@@ -66,6 +66,8 @@ def _bind(lib):
     lib.sama_oracle_losses.restype = None
     lib.sama_oracle_fd.argtypes = [C.c_int32, dp, dp, fp, C.c_double, C.c_int32, dp]
     lib.sama_oracle_fd.restype = None
+    lib.sama_oracle_meta_grad.argtypes = [C.c_int32, ip, fp, fp, ip, C.c_int32, dp]
+    lib.sama_oracle_meta_grad.restype = C.c_double
     lib.sama_oracle_step.argtypes = [C.c_int32, ip, C.c_int64, fp, fp, fp, fp, fp, ap, C.c_double,
                                      fp, ip, fp, C.c_int32, C.c_int32, dp, dp, dp, dp, dp, dp, dp]
     lib.sama_oracle_step.restype = C.c_int
@@ -146,6 +148,16 @@ def losses(dims: Sequence[int], theta, X, y, want_logits: bool = False):
                                _p(X, C.c_float), _p(y, C.c_int32), B, _p(out, C.c_double),
                                _p(logits, C.c_double))
     return (out, logits) if want_logits else out
+
+
+def meta_grad(dims: Sequence[int], theta, X, y):
+    """Direct gradient (Eq. 1): (L_meta, dL_meta/dtheta) of the mean cross-entropy on a clean batch, in double."""
+    dims_a = _i32(dims)
+    theta, X, y = _f32(theta), _f32(X), _i32(y)
+    g = np.empty(theta.size, dtype=np.float64)
+    loss = _load().sama_oracle_meta_grad(len(dims_a) - 1, _p(dims_a, C.c_int32), _p(theta, C.c_float),
+                                         _p(X, C.c_float), _p(y, C.c_int32), y.size, _p(g, C.c_double))
+    return float(loss), g
 
 
 def fd(loss_plus, loss_minus, lam, eps_fd: float, B_norm: int) -> np.ndarray:

@@ -157,6 +157,64 @@ void sama_oracle_losses(int32_t n_layers, const int32_t* dims, const double* the
     }
 }
 
+// Direct gradient -- the first factor of Eq. 1, dL_meta/dtheta, for the meta objective of Sec. 4.1:
+// L_meta(theta) = (1/B) sum_i CE(f(x_i; theta), y_i) on a clean batch.  Plain reverse-mode
+// differentiation of the same MLP, layer by layer:
+//   dz_L = (softmax(z_L) - onehot(y)) / B,
+//   dW_l = dz_l h_{l-1}^T,  db_l = dz_l,  dh_{l-1} = W_l^T dz_l,  dz_{l-1} = dh_{l-1} * [z_{l-1} > 0].
+// Returns L_meta; grad_out has the layout of theta.
+double sama_oracle_meta_grad(int32_t n_layers, const int32_t* dims, const float* theta, const float* X,
+                             const int32_t* y, int32_t B, double* grad_out) {
+    int64_t n = 0;
+    std::vector<int64_t> woff(n_layers), boff(n_layers);
+    for (int32_t l = 0; l < n_layers; ++l) {
+        woff[l] = n;
+        n += (int64_t)dims[l] * dims[l + 1];
+        boff[l] = n;
+        n += dims[l + 1];
+    }
+    for (int64_t k = 0; k < n; ++k) grad_out[k] = 0.0;
+    std::vector<std::vector<double>> h(n_layers + 1);  // h[l] = input of layer l (post-ReLU), h[L] = logits
+    for (int32_t l = 0; l <= n_layers; ++l) h[l].resize(dims[l]);
+    double loss = 0.0;
+    const int32_t C = dims[n_layers];
+    for (int32_t i = 0; i < B; ++i) {
+        for (int32_t k = 0; k < dims[0]; ++k) h[0][k] = (double)X[(int64_t)i * dims[0] + k];
+        for (int32_t l = 0; l < n_layers; ++l) {
+            const int32_t din = dims[l], dout = dims[l + 1];
+            for (int32_t j = 0; j < dout; ++j) {
+                double acc = (double)theta[boff[l] + j];
+                for (int32_t k = 0; k < din; ++k) acc += (double)theta[woff[l] + (int64_t)j * din + k] * h[l][k];
+                const bool hidden = l + 1 < n_layers;
+                h[l + 1][j] = (hidden && acc < 0.0) ? 0.0 : acc;
+            }
+        }
+        double zmax = h[n_layers][0];
+        for (int32_t c = 1; c < C; ++c) zmax = h[n_layers][c] > zmax ? h[n_layers][c] : zmax;
+        double se = 0.0;
+        for (int32_t c = 0; c < C; ++c) se += std::exp(h[n_layers][c] - zmax);
+        loss += (std::log(se) + zmax - h[n_layers][y[i]]) / (double)B;
+        std::vector<double> dz(C);
+        for (int32_t c = 0; c < C; ++c)
+            dz[c] = (std::exp(h[n_layers][c] - zmax) / se - (c == y[i] ? 1.0 : 0.0)) / (double)B;
+        for (int32_t l = n_layers - 1; l >= 0; --l) {
+            const int32_t din = dims[l], dout = dims[l + 1];
+            std::vector<double> dh(din, 0.0);
+            for (int32_t j = 0; j < dout; ++j) {
+                grad_out[boff[l] + j] += dz[j];
+                for (int32_t k = 0; k < din; ++k) {
+                    grad_out[woff[l] + (int64_t)j * din + k] += dz[j] * h[l][k];
+                    dh[k] += (double)theta[woff[l] + (int64_t)j * din + k] * dz[j];
+                }
+            }
+            if (l > 0)  // h[l] is a ReLU output: the derivative passes where it is positive
+                for (int32_t k = 0; k < din; ++k) dh[k] = h[l][k] > 0.0 ? dh[k] : 0.0;
+            dz.swap(dh);
+        }
+    }
+    return loss;
+}
+
 // S5 -- Eq. 5 for per-sample weight logits:
 // dL_base/dlambda_i = sigmoid'(lambda_i) loss_i / B_norm, hence
 // metagrad_i = -sigmoid'(lambda_i) (loss+_i - loss-_i) / (2 eps_fd B_norm).

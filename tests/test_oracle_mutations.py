@@ -29,6 +29,10 @@ MUTATIONS = {
     "fd_sign": ("metagrad_out[i] = -sg", "metagrad_out[i] = sg"),
     "fd_one_sided_scale": ("(2.0 * eps_fd * (double)B_norm)", "(eps_fd * (double)B_norm)"),
     "sigmoid_instead_of_derivative": ("-sg * (1.0 - sg) *", "-sg *"),
+    "meta_grad_relu_mask_dropped": ("dh[k] = h[l][k] > 0.0 ? dh[k] : 0.0;", "dh[k] = dh[k];"),
+    "meta_grad_no_onehot": ("(c == y[i] ? 1.0 : 0.0)", "0.0"),
+    "meta_grad_transposed_backprop": ("dh[k] += (double)theta[woff[l] + (int64_t)j * din + k] * dz[j];",
+                                      "dh[k] += (double)theta[woff[l] + ((int64_t)k * dout + j) % ((int64_t)din * dout)] * dz[j];"),
     "no_batch_mean": ("(2.0 * eps_fd * (double)B_norm)", "(2.0 * eps_fd)"),
 }
 

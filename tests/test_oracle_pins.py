@@ -359,3 +359,39 @@ def test_fd_sign_descends_meta_loss_direction():
     expect = -sg * (1 - sg) / B * np.dot(gd, gd)
     assert out["metagrad"][j] < 0
     assert out["metagrad"][j] == pytest.approx(expect, rel=1e-4)
+
+
+# ----------------------------------------------------------------------------
+# Direct gradient dL_meta/dtheta (first factor of Eq. 1)
+# ----------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dims,B", [((5, 3), 4), ((6, 5, 3), 7), ((4, 6, 5, 3), 5)])
+def test_meta_grad_matches_brute_force_differences(dims, B):
+    """Every component against a central difference of the mean cross-entropy (computed by the
+    forward pass, which has its own pins) in extended precision."""
+    cfg, w = W.custom_mlp(dims, B, seed=31)
+    theta = (w["theta"] + 0.1 * W.normal(31, 77, w["theta"].size).astype(np.float32)).astype(np.float32)
+    loss, g = oracle.meta_grad(dims, theta, w["X"], w["y"])
+    f = lambda t: numpy_losses(dims, t, np.asarray(w["X"], dtype=LD), w["y"], dtype=LD)[0].mean()
+    assert loss == pytest.approx(float(f(theta.astype(LD))), rel=1e-12)
+    ref = np.zeros(theta.size)
+    for k in range(theta.size):
+        e = np.zeros(theta.size, dtype=LD)
+        e[k] = LD(1e-6)
+        ref[k] = float((f(theta.astype(LD) + e) - f(theta.astype(LD) - e)) / LD(2e-6))
+    np.testing.assert_allclose(g, ref, rtol=1e-6, atol=1e-9)
+
+
+def test_meta_grad_single_layer_closed_form():
+    dims, B = (7, 4), 9
+    cfg, w = W.custom_mlp(dims, B, seed=33)
+    theta = w["theta"]
+    Wm, b = theta[:28].astype(np.float64).reshape(4, 7), theta[28:].astype(np.float64)
+    X = w["X"].astype(np.float64)
+    z = X @ Wm.T + b
+    sm = np.exp(z - z.max(1, keepdims=True))
+    sm /= sm.sum(1, keepdims=True)
+    sm[np.arange(B), w["y"]] -= 1
+    _, g = oracle.meta_grad(dims, theta, w["X"], w["y"])
+    np.testing.assert_allclose(g[:28].reshape(4, 7), sm.T @ X / B, rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(g[28:], sm.sum(0) / B, rtol=1e-12, atol=1e-15)
