@@ -219,6 +219,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--flat-n", type=int, default=0, help="override the length of a flat-vector workload")
+    ap.add_argument("--meta-grad", action="store_true",
+                    help="also time sama_meta_grad (the direct gradient that produces g_meta) on the same batch")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -391,6 +393,28 @@ def main():
         e2e = {"value": world * Ke / te, "unit": "steps/s", "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(4 * B + 4), "steps": Ke,
                "note": "sama_step_host: all inputs copied from pinned host memory every step"}
+    meta = None
+    if args.meta_grad and not flat:
+        gm_out = torch.empty(n, dtype=torch.float32, device=dev)
+        for _ in range(3):
+            S.sama_meta_grad(ctx, mlp, d["theta"], d["X"], d["y"], B, gm_out, None, stream)
+        Km = max(3, min(args.steps, 50))
+        evm = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(Km)]
+        sampler.active.set()
+        for a_, b_ in evm:
+            flush_buf.fill_(1)
+            a_.record(stream)
+            S.sama_meta_grad(ctx, mlp, d["theta"], d["X"], d["y"], B, gm_out, None, stream)
+            b_.record(stream)
+        torch.cuda.synchronize()
+        sampler.active.clear()
+        msm = sum(a_.elapsed_time(b_) for a_, b_ in evm) / Km
+        flops_m = 1.5 * cfg.forward_flops   # forward + dz W + dz^T h of ONE branch = 3/2 of the dual-branch forward
+        mhz = (sampler.summary()["sm_mhz"] or 1965.0)
+        peak_m = sm_count * FMA_LANES_PER_SM * 2 * mhz * 1e6 / 1e12
+        meta = {"ms_per_call": msm, "calls_per_s": 1e3 / msm, "tflops": flops_m / (msm * 1e-3) / 1e12,
+                "frac_of_fma_peak": flops_m / (msm * 1e-3) / 1e12 / peak_m, "peak_tflops": peak_m,
+                "note": "fp32 FMA, strided operands; algorithmic flops = 3 single-branch matrix products per layer"}
     sampler.stop_flag.set()
     clocks = sampler.summary()
 
@@ -402,6 +426,8 @@ def main():
                       "replicas": "one independent step per rank, no data-path collective"},
            "clocks": clocks, "gpu_launches": int(launches), "device_status": int(status),
            "wall_s_timed_region": t_wall, "roofline": roofline, "rooflines": rooflines, "kernels": per_kernel}
+    if meta:
+        out["meta_grad"] = meta
     if e2e:
         out["e2e"] = e2e
     if flat:

@@ -172,6 +172,16 @@ int sama_step(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* thet
               float* p_out, float* theta_plus, float* theta_minus, float* metagrad_out,
               float* loss_plus_out, float* loss_minus_out, void* stream);
 
+/* Direct gradient, the first factor of Eq. 1: g_meta = dL_meta/dtheta for the meta objective of
+ * Sec. 4.1, L_meta(theta) = (1/B) sum_i CE(f(x_i; theta), y_i) on a clean batch, by reverse
+ * differentiation of the same MLP (fp32).  Its output is the `g_meta` input of sama_adapt / sama_step.
+ * theta: [n_params(mlp)].  X_meta: [B][d_0].  y_meta: int32 [B].  g_meta_out: [n_params(mlp)], must not
+ * overlap the inputs.  loss_out: one float on the device (the mean loss), or NULL.  A label outside
+ * [0, d_L) sets SAMA_DEV_BAD_LABEL and that sample contributes nothing.  Needs a context created
+ * with an mlp whose layer widths are not smaller, B <= max_batch.  Results are reproducible bit for bit. */
+int sama_meta_grad(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta, const float* X_meta,
+                   const int32_t* y_meta, int32_t B, float* g_meta_out, float* loss_out, void* stream);
+
 /* sama_step (Fig. 2) for callers whose data lives in HOST memory: every
  * pointer below is a host pointer (pinned memory makes the copies
  * asynchronous).  Copies the inputs to staging buffers owned by the context
@@ -226,7 +236,9 @@ enum {
     SAMA_K_SPLIT = 5,
     SAMA_K_GEMM_TF32X3 = 6,
     SAMA_K_HEAD = 7, /* narrow last layer fused with cross-entropy + central difference */
-    SAMA_K_PERTURB_SPLIT = 8 /* perturbation that also writes the tensor-core operands of W+ and W- */
+    SAMA_K_PERTURB_SPLIT = 8, /* perturbation that also writes the tensor-core operands of W+ and W- */
+    SAMA_K_META_GEMM = 9,     /* matrix products of the direct gradient (forward, dz W, dz^T h) */
+    SAMA_K_META_AUX = 10      /* softmax gradient, bias sums, mean loss of the direct gradient */
 };
 typedef struct sama_kernel_time_t {
     int32_t kind;  /* SAMA_K_* */

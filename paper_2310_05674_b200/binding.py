@@ -47,7 +47,7 @@ class sama_kernel_time_t(C.Structure):
 
 
 KERNEL_KINDS = {0: "adapt_sumsq", 1: "sumsq", 2: "perturb", 3: "gemm_ffma", 4: "ce_fd", 5: "split_tf32",
-                6: "gemm_tf32x3", 7: "head_ce_fd", 8: "perturb_split"}
+                6: "gemm_tf32x3", 7: "head_ce_fd", 8: "perturb_split", 9: "meta_gemm", 10: "meta_aux"}
 
 
 class sama_mlp_t(C.Structure):
@@ -92,6 +92,7 @@ lib.sama_fd_metagrad.argtypes = [_vp, C.POINTER(sama_mlp_t), _vp, _vp, _vp, _vp,
                                  _vp, _vp]
 lib.sama_step.argtypes = [_vp, C.POINTER(sama_mlp_t), C.c_int64, _vp, _vp, _vp, _vp, _vp, C.POINTER(sama_adam_t),
                           C.c_float, _vp, _vp, _vp, C.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.sama_meta_grad.argtypes = [_vp, C.POINTER(sama_mlp_t), _vp, _vp, _vp, C.c_int32, _vp, _vp, _vp]
 lib.sama_step_host.argtypes = [_vp, C.POINTER(sama_mlp_t), C.c_int64, _vp, _vp, _vp, _vp, _vp,
                                C.POINTER(sama_adam_t), C.c_float, _vp, _vp, _vp, C.c_int32, _vp, _vp, _vp, _vp]
 lib.sama_ctx_sumsq.argtypes = [_vp]
@@ -190,6 +191,11 @@ def sama_step(ctx, mlp: MLP, n, theta, m, s, g_base, g_meta, adam: Adam, alpha, 
                                 C.byref(a), float(alpha), _ptr(X), _ptr(y), _ptr(lam), int(B), _ptr(p_out),
                                 _ptr(theta_plus), _ptr(theta_minus), _ptr(metagrad_out), _ptr(loss_plus_out),
                                 _ptr(loss_minus_out), _stream(stream)), "sama_step")
+
+
+def sama_meta_grad(ctx, mlp: MLP, theta, X_meta, y_meta, B, g_meta_out, loss_out=None, stream=None) -> int:
+    return _check(lib.sama_meta_grad(ctx, mlp.c(), _ptr(theta), _ptr(X_meta), _ptr(y_meta), int(B),
+                                     _ptr(g_meta_out), _ptr(loss_out), _stream(stream)), "sama_meta_grad")
 
 
 def sama_step_host(ctx, mlp: MLP, n, theta_host, m_host, s_host, g_base_host, g_meta_host, adam: Adam, alpha,

@@ -383,6 +383,8 @@ int sama_create(sama_ctx** out, int device, int64_t max_n, int32_t max_batch, co
         ctx->a_split_half = 2 * (size_t)max_batch * amax;
         ok = ok && cudaMalloc(&ctx->x_split, sizeof(float) * 2 * ctx->x_split_half) == cudaSuccess &&
              cudaMalloc(&ctx->w_split, sizeof(float) * 2 * ctx->w_split_half) == cudaSuccess;
+        ctx->mg_ws_floats = meta_grad_workspace_floats(mlp, max_batch);
+        ok = ok && cudaMalloc(&ctx->mg_ws, sizeof(float) * ctx->mg_ws_floats) == cudaSuccess;
         ctx->tc_ws_floats = (size_t)8 << 20;  // 32 MiB of split-K partial tiles
         ok = ok && cudaMalloc(&ctx->tc_ws, sizeof(float) * ctx->tc_ws_floats) == cudaSuccess &&
              cudaMalloc(&ctx->tc_counters, sizeof(int) * kTcCounters) == cudaSuccess &&
@@ -413,6 +415,7 @@ int sama_destroy(sama_ctx* ctx) {
     cudaFree(ctx->a_split[0]);
     cudaFree(ctx->a_split[1]);
     cudaFree(ctx->tc_ws);
+    cudaFree(ctx->mg_ws);
     cudaFree(ctx->tc_counters);
     cudaFree(ctx->stage);
     if (ctx->prof) {
@@ -527,6 +530,27 @@ int sama_step(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* thet
                                       nullptr, st));
     return run_fd(ctx, mlp, theta_plus, theta_minus, X, y, lambda, B, nullptr, metagrad_out, loss_plus_out,
                   loss_minus_out, st, fused, x_fused);
+}
+
+int sama_meta_grad(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta, const float* X_meta,
+                   const int32_t* y_meta, int32_t B, float* g_meta_out, float* loss_out, void* stream) {
+    if (!ctx || !theta || !X_meta || !y_meta || !g_meta_out) return SAMA_ERR_NULL;
+    const int rc = check_mlp(mlp);
+    if (rc != SAMA_OK) return rc;
+    if (B < 1 || B > ctx->max_batch || !ctx->mg_ws) return SAMA_ERR_SIZE;
+    if (meta_grad_workspace_floats(mlp, B) > ctx->mg_ws_floats) return SAMA_ERR_SIZE;
+    if (!aligned(theta, 4) || !aligned(X_meta, 4) || !aligned(y_meta, 4) || !aligned(g_meta_out, 4) ||
+        !aligned(loss_out, 4))
+        return SAMA_ERR_ALIGN;
+    const size_t nb = (size_t)sama_mlp_param_count(mlp) * 4, bb = (size_t)B * 4;
+    if (overlaps(g_meta_out, nb, theta, nb) || overlaps(g_meta_out, nb, X_meta, (size_t)B * mlp->dims[0] * 4) ||
+        overlaps(g_meta_out, nb, y_meta, bb) || overlaps(g_meta_out, nb, loss_out, 4) ||
+        overlaps(loss_out, 4, theta, nb) || overlaps(loss_out, 4, X_meta, (size_t)B * mlp->dims[0] * 4))
+        return SAMA_ERR_OVERLAP;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SAMA_ERR_CUDA;
+    SAMA_CUDA(ctx, run_meta_grad(ctx, mlp, theta, X_meta, y_meta, B, g_meta_out, loss_out, (cudaStream_t)stream));
+    return SAMA_OK;
 }
 
 int sama_step_host(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* theta_host, const float* m_host,

@@ -89,6 +89,8 @@ struct sama_ctx {
     float* tc_ws;                  // device: split-K partial tiles of the tensor-core path
     size_t tc_ws_floats;
     int* tc_counters;              // device [kTcCounters], zero between launches
+    float* mg_ws;                  // device: workspace of the direct gradient (activations, dz, losses)
+    size_t mg_ws_floats;
     float* stage;                  // device: staging of the host entry point (allocated on first use)
     size_t stage_bytes;
     sama::Profiler* prof;          // host
@@ -221,5 +223,10 @@ cudaError_t launch_head_ce_fd(sama_ctx* ctx, const float* h_plus, const float* h
                               const float* w_plus, const float* w_minus, const float* b_plus, const float* b_minus,
                               const int32_t* y, const float* lambda, int B, int C, int K, const float* eps_fd,
                               float* metagrad, float* loss_plus, float* loss_minus, cudaStream_t st);
+
+// meta_grad.cu : direct gradient dL_meta/dtheta (Eq. 1)
+size_t meta_grad_workspace_floats(const sama_mlp_t* mlp, int64_t B);
+cudaError_t run_meta_grad(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta, const float* X, const int32_t* y,
+                          int32_t B, float* g_out, float* loss_out, cudaStream_t st);
 
 }  // namespace sama
