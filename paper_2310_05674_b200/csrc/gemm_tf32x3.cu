@@ -192,6 +192,9 @@ struct TcArgs {
     int M, N, num_kb;
     int ldc, ld_next;      // ld_next = N rounded up to 32 (zero-filled tail)
     int relu, last, shared_a;
+    int both;              // hidden layer that also stores its fp32 result (kept for a backward pass)
+    const float* mask;     // [M][ldm] or null: results are zeroed where mask <= 0
+    int ldm;
     int tiles_m, tiles_n, group_n;
     int splits, kb_per_split;  // split-K: grid.z = 2 * splits, each CTA takes kb_per_split k-blocks
     float* ws;                 // split-K partial tiles [2 * tiles][splits][BM][BN]
@@ -420,11 +423,17 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                 if (m < args.M) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
-                        float x = v[j] + ((n + j < args.N) ? bias[n + j] : 0.f);
+                        float x = v[j] + ((bias != nullptr && n + j < args.N) ? bias[n + j] : 0.f);
                         if (args.relu && x < 0.f) x = 0.f;
                         v[j] = x;
                     }
-                    if (args.last) {
+                    if (args.mask) {  // backward pass: the derivative passes only where the forward activation was positive
+                        const float* mk = args.mask + (int64_t)m * args.ldm + n;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (n + j < args.N && !(mk[j] > 0.f)) v[j] = 0.f;
+                    }
+                    if (args.last || args.both) {
                         float* dst = (br ? args.out_f32[1] : args.out_f32[0]) + (int64_t)m * args.ldc + n;
                         if (n + 15 < args.N && (args.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
 #pragma unroll
@@ -436,7 +445,8 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                             for (int j = 0; j < 16; ++j)
                                 if (n + j < args.N) dst[j] = v[j];
                         }
-                    } else if (n < args.ld_next) {
+                    }
+                    if (!args.last && n < args.ld_next) {
                         // columns in [N, ld_next) are the next layer's zero padding along K
                         const int64_t off = ((int64_t)br * args.M + m) * args.ld_next + n;
                         float hi[16], lo[16];
@@ -518,6 +528,37 @@ split_tf32_kernel(SplitArgs a) {
     }
 }
 
+// hi / lo of the transpose: src [rows][cols] -> out [cols][ld_out], ld_out = rows rounded up to 32, zero padded.
+// 32 x 32 tiles through shared memory so that both the read and the writes are coalesced.
+__global__ void __launch_bounds__(256)
+split_transpose_tf32_kernel(const float* __restrict__ src, int64_t rows, int cols, int ld_out,
+                            float* __restrict__ hi, float* __restrict__ lo) {
+    pdl_trigger();
+    pdl_wait();
+    __shared__ float tile[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;  // 32 x 8
+    const int64_t r0 = (int64_t)blockIdx.y * 32;
+    const int c0 = blockIdx.x * 32;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int64_t r = r0 + ty + 8 * i;
+        const int c = c0 + tx;
+        tile[ty + 8 * i][tx] = (r < rows && c < cols) ? src[r * cols + c] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int c = c0 + ty + 8 * i;       // output row
+        const int64_t r = r0 + tx;           // output column (< ld_out: the grid covers ld_out / 32 tiles)
+        if (c < cols) {
+            const float x = tile[tx][ty + 8 * i];
+            const float h = to_tf32(x);
+            hi[(int64_t)c * ld_out + r] = h;
+            lo[(int64_t)c * ld_out + r] = to_tf32(x - h);
+        }
+    }
+}
+
 // ------------------------------------------------------------------ host side
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -591,6 +632,14 @@ cudaError_t launch_split_tf32(sama_ctx* ctx, const float* src0, const float* src
                : launch_dependent(split_tf32_kernel<false>, grid, dim3(256), 0, st, a);
 }
 
+cudaError_t launch_split_transpose_tf32(sama_ctx* ctx, const float* src, int64_t rows, int cols, float* hi, float* lo,
+                                        cudaStream_t st) {
+    const int ld_out = round_up32((int)rows);
+    dim3 grid((cols + 31) / 32, ld_out / 32, 1);
+    KernelScope scope(ctx, SAMA_K_SPLIT, -1, st);
+    return launch_dependent(split_transpose_tf32_kernel, grid, dim3(256), 0, st, src, rows, cols, ld_out, hi, lo);
+}
+
 // One layer on the tensor cores.  a_hi/a_lo: [shared_a ? 1 : 2][M][Kp]; w_hi/w_lo: [2][N][Kp]; Kp = K rounded
 // up to 32.  Hidden layers write the next operands (out_hi/out_lo, [2][M][round_up32(N)]); the last layer
 // writes fp32 logits.
@@ -598,7 +647,8 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     const int Kp = round_up32(L.K);
     // N-tile: 16 for a narrow last layer; 64 when 128-wide tiles would leave SMs idle; else 128.
     // (Hidden layers never take 16: their tiles must also write the zero padding up to round_up32(N).)
-    const int64_t tiles128 = (int64_t)((L.M + BM - 1) / BM) * ((L.N + 127) / 128) * 2;
+    const int nbr = L.branches == 1 ? 1 : 2;  // the direct gradient runs a single branch
+    const int64_t tiles128 = (int64_t)((L.M + BM - 1) / BM) * ((L.N + 127) / 128) * nbr;
     // Split-K (several CTAs per tile, partials added in split order by the last CTA to arrive) exists for
     // contractions that are long relative to the grid, but measured slower than 64-wide tiles on every
     // workload here (the partial-tile round trip costs more than the idle SMs), so it is off unless the
@@ -609,7 +659,7 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     const int num_kb_total = Kp / BKF;
     int splits = 1;
     {
-        const int64_t tiles = (int64_t)((L.M + BM - 1) / BM) * ((L.N + bn - 1) / bn) * 2;
+        const int64_t tiles = (int64_t)((L.M + BM - 1) / BM) * ((L.N + bn - 1) / bn) * nbr;
         int want = 1;
         if (const char* e = std::getenv("SAMA_TC_SPLITS")) want = std::atoi(e);
         if (want > 8) want = 8;
@@ -625,7 +675,7 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     bool pair = !narrow_last && splits == 1 && L.M > BM && L.N >= 128;
     if (const char* e = std::getenv("SAMA_TC_PAIR")) pair = pair && std::atoi(e) != 0;
     if (pair) {
-        auto ctas = [&](int w) { return 2 * (int64_t)((L.M + 2 * BM - 1) / (2 * BM)) * ((L.N + w - 1) / w) * 2; };
+        auto ctas = [&](int w) { return 2 * (int64_t)((L.M + 2 * BM - 1) / (2 * BM)) * ((L.N + w - 1) / w) * nbr; };
         int pbn = 0;
         if (L.N >= 256 && ctas(256) >= ctx->sm_count) pbn = 256;
         else if (ctas(128) >= ctx->sm_count) pbn = 128;
@@ -633,7 +683,7 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
         if (pbn == 0 || L.N < pbn) pair = false; else bn = pbn;
     }
     CUtensorMap maps[4];
-    const int a_slabs = L.shared_a ? 1 : 2;
+    const int a_slabs = (L.shared_a || nbr == 1) ? 1 : 2;
     // a box never exceeds the tensor's extent; rows of the shared-memory tile that no copy fills only
     // feed output rows / columns that the epilogue does not store
     const int wrows = pair ? bn / 2 : bn;
@@ -641,7 +691,8 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     const int64_t a_slab = (int64_t)L.M * Kp;
     if (!make_map(&maps[0], L.a_hi, Kp, L.M, a_slabs, a_box, a_slab) ||
         !make_map(&maps[1], L.a_lo, Kp, L.M, a_slabs, a_box, a_slab) ||
-        !make_map(&maps[2], L.w_hi, Kp, L.N, 2, w_box, L.w_slab) || !make_map(&maps[3], L.w_lo, Kp, L.N, 2, w_box, L.w_slab))
+        !make_map(&maps[2], L.w_hi, Kp, L.N, nbr, w_box, L.w_slab) ||
+        !make_map(&maps[3], L.w_lo, Kp, L.N, nbr, w_box, L.w_slab))
         return cudaErrorInvalidValue;
     TcArgs a;
     a.bias[0] = L.bias[0];
@@ -658,6 +709,9 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     a.relu = L.relu;
     a.last = L.last;
     a.shared_a = L.shared_a;
+    a.both = L.both;
+    a.mask = L.mask;
+    a.ldm = L.ldm;
     a.tx_bytes = (uint32_t)(2 * a_box * BKF * 4 + 2 * w_box * BKF * 4) * (pair ? 2u : 1u);  // a pair's barrier counts both CTAs' copies
     a.status = &ctx->scalars->status;
     a.tiles_m = pair ? (L.M + 2 * BM - 1) / (2 * BM) : (L.M + BM - 1) / BM;
@@ -671,7 +725,7 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     if (a.group_n < 1) a.group_n = 1;
     if (a.group_n > a.tiles_n) a.group_n = a.tiles_n;
     if (const char* e = std::getenv("SAMA_TC_GROUP")) { const int g = std::atoi(e); if (g >= 1 && g <= a.tiles_n) a.group_n = g; }
-    dim3 grid(a.tiles_m * a.tiles_n * (pair ? 2 : 1), 1, 2 * a.splits);
+    dim3 grid(a.tiles_m * a.tiles_n * (pair ? 2 : 1), 1, nbr * a.splits);
     KernelScope scope(ctx, SAMA_K_GEMM_TF32X3, L.layer, st);
     if (pair) {
         if (bn == 64) return launch_tc<64, true>(maps, a, grid, st);

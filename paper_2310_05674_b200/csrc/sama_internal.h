@@ -207,7 +207,14 @@ struct TcLayer {
     float* out_lo;
     int M, N, K, ldc;
     int relu, last, shared_a, layer;
+    int branches = 2;            // 1: only branch 0 (the direct gradient)
+    int both = 0;                // hidden layer that also stores fp32 to out_f32
+    const float* mask = nullptr; // [M][ldm]: zero the result where mask <= 0
+    int ldm = 0;
 };
+// hi/lo of the TRANSPOSE of a dense fp32 matrix [rows][cols]: out [cols][round32(rows)], zero padded
+cudaError_t launch_split_transpose_tf32(sama_ctx* ctx, const float* src, int64_t rows, int cols, float* hi, float* lo,
+                                        cudaStream_t st);
 cudaError_t launch_split_tf32(sama_ctx* ctx, const float* src0, const float* src1, int branches, int64_t rows,
                               int cols, float* hi, float* lo, int64_t slab, cudaStream_t st);
 cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st);
