@@ -410,11 +410,18 @@ def main():
         sampler.active.clear()
         msm = sum(a_.elapsed_time(b_) for a_, b_ in evm) / Km
         flops_m = 1.5 * cfg.forward_flops   # forward + dz W + dz^T h of ONE branch = 3/2 of the dual-branch forward
-        mhz = (sampler.summary()["sm_mhz"] or 1965.0)
-        peak_m = sm_count * FMA_LANES_PER_SM * 2 * mhz * 1e6 / 1e12
-        meta = {"ms_per_call": msm, "calls_per_s": 1e3 / msm, "tflops": flops_m / (msm * 1e-3) / 1e12,
-                "frac_of_fma_peak": flops_m / (msm * 1e-3) / 1e12 / peak_m, "peak_tflops": peak_m,
-                "note": "fp32 FMA, strided operands; algorithmic flops = 3 single-branch matrix products per layer"}
+        if args.gemm_mode == 1:
+            mhz = (sampler.summary()["sm_mhz"] or 1965.0)
+            peak_m = sm_count * FMA_LANES_PER_SM * 2 * mhz * 1e6 / 1e12
+            bound_m, src_m = "alu", "%d SMs x 128 FMA lanes x 2 x %.0f MHz" % (sm_count, mhz)
+        else:
+            peak_m = peaks["bf16_tflops_sustained"] * 0.5 / 3.0
+            bound_m, src_m = "tensor", peaks["source"] + " sustained bf16 x 0.5 / 3 products per fp32-faithful product"
+        ach_m = flops_m / (msm * 1e-3) / 1e12
+        meta = {"ms_per_call": msm, "calls_per_s": 1e3 / msm, "bound": bound_m, "achieved": ach_m, "peak": peak_m,
+                "unit": "TFLOP/s", "frac": ach_m / peak_m, "peak_source": src_m,
+                "note": "algorithmic flops = 3 single-branch matrix products per layer (forward, dz W, dz^T h); "
+                        "time includes the operand split / transpose kernels"}
     sampler.stop_flag.set()
     clocks = sampler.summary()
 

@@ -192,8 +192,160 @@ size_t meta_grad_workspace_floats(const sama_mlp_t* mlp, int64_t B) {
     return (size_t)B * (acts + 2 * widest + 1);
 }
 
-cudaError_t run_meta_grad(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta, const float* X, const int32_t* y,
-                          int32_t B, float* g_out, float* loss_out, cudaStream_t st) {
+namespace {
+
+inline size_t r32(size_t x) { return (x + 31) & ~(size_t)31; }
+
+// Operand buffers of the tensor-core path (floats; each region holds hi then lo).
+struct TcPlan {
+    size_t dzs;    // dz split            [B][r32(widest)]
+    size_t wt;     // W_l^T split          [d_{l-1}][r32(d_l)], largest layer
+    size_t tz;     // dz^T split           [widest][r32(B)]
+    size_t th;     // h^T split            [widest][r32(B)]
+    size_t total;
+    size_t half_dzs, half_wt, half_t;
+};
+TcPlan tc_plan(const sama_mlp_t* mlp, int64_t B) {
+    size_t widest = 0, wt = 0;
+    for (int l = 0; l <= mlp->n_layers; ++l) widest = (size_t)mlp->dims[l] > widest ? (size_t)mlp->dims[l] : widest;
+    for (int l = 0; l < mlp->n_layers; ++l) {
+        const size_t e = (size_t)mlp->dims[l] * r32(mlp->dims[l + 1]);
+        wt = e > wt ? e : wt;
+    }
+    TcPlan p;
+    p.half_dzs = (size_t)B * r32(widest);
+    p.half_wt = wt;
+    p.half_t = widest * r32((size_t)B);
+    p.dzs = 0;
+    p.wt = p.dzs + 2 * p.half_dzs;
+    p.tz = p.wt + 2 * p.half_wt;
+    p.th = p.tz + 2 * p.half_t;
+    p.total = p.th + 2 * p.half_t;
+    return p;
+}
+
+}  // namespace
+
+size_t meta_grad_tc_floats(const sama_mlp_t* mlp, int64_t B) { return tc_plan(mlp, B).total; }
+
+// Same computation with every matrix product on the tensor cores (three TF32 products per fp32 product,
+// as in the forward pass of the step): operands are split, and transposed where the contraction runs
+// over the batch or the outputs, by small HBM-bound kernels.
+static cudaError_t run_meta_grad_tc(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta, const float* X,
+                                    const int32_t* y, int32_t B, float* g_out, float* loss_out, cudaStream_t st) {
+    const int L = mlp->n_layers;
+    const SplitLayout lay = make_split_layout(mlp);
+    const TcPlan plan = tc_plan(mlp, B);
+    size_t widest = 0;
+    for (int l = 0; l <= L; ++l) widest = (size_t)mlp->dims[l] > widest ? (size_t)mlp->dims[l] : widest;
+    // fp32 workspace: kept activations, dz ping-pong, losses (same carving as the FMA path)
+    float* cur = ctx->mg_ws;
+    const float* h[kMaxLayers + 1];
+    float* hbuf[kMaxLayers + 1];
+    h[0] = X;
+    for (int l = 1; l <= L; ++l) {
+        hbuf[l] = cur;
+        h[l] = cur;
+        cur += (size_t)B * mlp->dims[l];
+    }
+    float* dzb[2] = {cur, cur + (size_t)B * widest};
+    float* losses = cur + 2 * (size_t)B * widest;
+    float* tc = ctx->mg_tc;
+    float* w_hi = ctx->w_split;
+    float* w_lo = ctx->w_split + ctx->w_split_half;
+    cudaError_t e;
+    // forward: operands of theta and X, then one single-branch product per layer that keeps fp32 and
+    // writes the next operand
+    if ((e = launch_split_tf32(ctx, X, X, 1, B, mlp->dims[0], ctx->x_split, ctx->x_split + ctx->x_split_half, 0, st)) !=
+        cudaSuccess)
+        return e;
+    for (int l = 0; l < L; ++l) {
+        const int din = mlp->dims[l], dout = mlp->dims[l + 1];
+        const bool last = (l + 1 == L);
+        if ((e = launch_split_tf32(ctx, theta + lay.w_off[l], theta + lay.w_off[l], 1, dout, din, w_hi + lay.s_off[l],
+                                   w_lo + lay.s_off[l], lay.slab, st)) != cudaSuccess)
+            return e;
+        TcLayer t;
+        t.a_hi = l == 0 ? ctx->x_split : ctx->a_split[(l - 1) & 1];
+        t.a_lo = l == 0 ? ctx->x_split + ctx->x_split_half : ctx->a_split[(l - 1) & 1] + ctx->a_split_half;
+        t.w_hi = w_hi + lay.s_off[l];
+        t.w_lo = w_lo + lay.s_off[l];
+        t.w_slab = (int64_t)dout * lay.Kp[l];
+        t.bias[0] = t.bias[1] = theta + lay.w_off[l] + lay.w_cnt[l];
+        t.out_f32[0] = t.out_f32[1] = hbuf[l + 1];
+        t.out_hi = last ? nullptr : ctx->a_split[l & 1];
+        t.out_lo = last ? nullptr : ctx->a_split[l & 1] + ctx->a_split_half;
+        t.M = B; t.N = dout; t.K = din; t.ldc = dout;
+        t.relu = last ? 0 : 1; t.last = last ? 1 : 0; t.shared_a = 1; t.layer = l;
+        t.branches = 1; t.both = last ? 0 : 1;
+        if ((e = launch_gemm_tf32x3(ctx, t, st)) != cudaSuccess) return e;
+    }
+    const int C = mlp->dims[L];
+    {
+        KernelScope scope(ctx, SAMA_K_META_AUX, -1, st);
+        if ((e = launch_dependent(softmax_grad_kernel, dim3((B + 3) / 4), dim3(128), 0, st, hbuf[L], y, (int)B, C,
+                                  losses, ctx->scalars)) != cudaSuccess)
+            return e;
+    }
+    if (loss_out) {
+        KernelScope scope(ctx, SAMA_K_META_AUX, -1, st);
+        if ((e = launch_dependent(mean_kernel, dim3(1), dim3(256), 0, st, (const float*)losses, (int)B, loss_out)) !=
+            cudaSuccess)
+            return e;
+    }
+    const float* dz = hbuf[L];
+    const int Bp = (int)r32((size_t)B);
+    for (int l = L - 1; l >= 0; --l) {
+        const int din = mlp->dims[l], dout = mlp->dims[l + 1];
+        // dW[dout][din] = dz^T h_{l}: both operands transposed so that the batch is the contraction index
+        if ((e = launch_split_transpose_tf32(ctx, dz, B, dout, tc + plan.tz, tc + plan.tz + plan.half_t, st)) != cudaSuccess)
+            return e;
+        if ((e = launch_split_transpose_tf32(ctx, h[l], B, din, tc + plan.th, tc + plan.th + plan.half_t, st)) != cudaSuccess)
+            return e;
+        TcLayer tw;
+        tw.a_hi = tc + plan.tz; tw.a_lo = tc + plan.tz + plan.half_t;
+        tw.w_hi = tc + plan.th; tw.w_lo = tc + plan.th + plan.half_t;
+        tw.w_slab = (int64_t)din * Bp;
+        tw.bias[0] = tw.bias[1] = nullptr;
+        tw.out_f32[0] = tw.out_f32[1] = g_out + lay.w_off[l];
+        tw.out_hi = tw.out_lo = nullptr;
+        tw.M = dout; tw.N = din; tw.K = B; tw.ldc = din;
+        tw.relu = 0; tw.last = 1; tw.shared_a = 1; tw.layer = l; tw.branches = 1;
+        if ((e = launch_gemm_tf32x3(ctx, tw, st)) != cudaSuccess) return e;
+        {
+            KernelScope scope(ctx, SAMA_K_META_AUX, l, st);
+            if ((e = launch_dependent(colsum_kernel, dim3((dout + 255) / 256), dim3(256), 0, st, dz, (int)B, dout,
+                                      g_out + lay.w_off[l] + lay.w_cnt[l])) != cudaSuccess)
+                return e;
+        }
+        if (l > 0) {
+            // dz_{l-1}[B][din] = (dz W_l) masked by h_l > 0: W_l transposed so that its outputs are the contraction index
+            if ((e = launch_split_tf32(ctx, dz, dz, 1, B, dout, tc + plan.dzs, tc + plan.dzs + plan.half_dzs, 0, st)) !=
+                cudaSuccess)
+                return e;
+            if ((e = launch_split_transpose_tf32(ctx, theta + lay.w_off[l], dout, din, tc + plan.wt,
+                                                 tc + plan.wt + plan.half_wt, st)) != cudaSuccess)
+                return e;
+            TcLayer th_;
+            th_.a_hi = tc + plan.dzs; th_.a_lo = tc + plan.dzs + plan.half_dzs;
+            th_.w_hi = tc + plan.wt; th_.w_lo = tc + plan.wt + plan.half_wt;
+            th_.w_slab = (int64_t)din * (int64_t)r32((size_t)dout);
+            th_.bias[0] = th_.bias[1] = nullptr;
+            float* out = dzb[l & 1];
+            th_.out_f32[0] = th_.out_f32[1] = out;
+            th_.out_hi = th_.out_lo = nullptr;
+            th_.M = B; th_.N = din; th_.K = dout; th_.ldc = din;
+            th_.relu = 0; th_.last = 1; th_.shared_a = 1; th_.layer = l; th_.branches = 1;
+            th_.mask = h[l]; th_.ldm = din;
+            if ((e = launch_gemm_tf32x3(ctx, th_, st)) != cudaSuccess) return e;
+            dz = out;
+        }
+    }
+    return cudaSuccess;
+}
+
+static cudaError_t run_meta_grad_fma(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta, const float* X,
+                                     const int32_t* y, int32_t B, float* g_out, float* loss_out, cudaStream_t st) {
     const int L = mlp->n_layers;
     size_t widest = 0;
     for (int l = 0; l <= L; ++l) widest = (size_t)mlp->dims[l] > widest ? (size_t)mlp->dims[l] : widest;
@@ -276,6 +428,18 @@ cudaError_t run_meta_grad(sama_ctx* ctx, const sama_mlp_t* mlp, const float* the
         }
     }
     return cudaSuccess;
+}
+
+// Tensor cores unless the context is in fp32-FMA mode or the model does not fit the operand workspaces.
+cudaError_t run_meta_grad(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta, const float* X, const int32_t* y,
+                          int32_t B, float* g_out, float* loss_out, cudaStream_t st) {
+    const int L = mlp->n_layers;
+    bool fits = ctx->gemm_mode != 1 && ctx->mg_tc && tc_plan(mlp, B).total <= ctx->mg_tc_floats &&
+                ctx->x_split_half >= (size_t)B * r32(mlp->dims[0]) &&
+                (size_t)make_split_layout(mlp).slab <= ctx->w_split_half;
+    for (int l = 0; l + 1 < L && fits; ++l) fits = 2 * (size_t)B * r32(mlp->dims[l + 1]) <= ctx->a_split_half * 2;
+    if (fits) return run_meta_grad_tc(ctx, mlp, theta, X, y, B, g_out, loss_out, st);
+    return run_meta_grad_fma(ctx, mlp, theta, X, y, B, g_out, loss_out, st);
 }
 
 }  // namespace sama

@@ -154,6 +154,9 @@ int validate_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, c
     return SAMA_OK;
 }
 
+}  // namespace
+
+namespace sama {
 SplitLayout make_split_layout(const sama_mlp_t* mlp) {
     SplitLayout lay;
     std::memset(&lay, 0, sizeof(lay));
@@ -172,6 +175,10 @@ SplitLayout make_split_layout(const sama_mlp_t* mlp) {
     lay.slab = soff;
     return lay;
 }
+
+}  // namespace sama
+
+namespace {
 
 // Whether this model fits the operand-split workspace of the tensor-core path.
 bool tc_fits(const sama_ctx* ctx, const sama_mlp_t* mlp, int32_t B) {
@@ -385,6 +392,8 @@ int sama_create(sama_ctx** out, int device, int64_t max_n, int32_t max_batch, co
              cudaMalloc(&ctx->w_split, sizeof(float) * 2 * ctx->w_split_half) == cudaSuccess;
         ctx->mg_ws_floats = meta_grad_workspace_floats(mlp, max_batch);
         ok = ok && cudaMalloc(&ctx->mg_ws, sizeof(float) * ctx->mg_ws_floats) == cudaSuccess;
+        ctx->mg_tc_floats = meta_grad_tc_floats(mlp, max_batch);
+        ok = ok && cudaMalloc(&ctx->mg_tc, sizeof(float) * ctx->mg_tc_floats) == cudaSuccess;
         ctx->tc_ws_floats = (size_t)8 << 20;  // 32 MiB of split-K partial tiles
         ok = ok && cudaMalloc(&ctx->tc_ws, sizeof(float) * ctx->tc_ws_floats) == cudaSuccess &&
              cudaMalloc(&ctx->tc_counters, sizeof(int) * kTcCounters) == cudaSuccess &&
@@ -416,6 +425,7 @@ int sama_destroy(sama_ctx* ctx) {
     cudaFree(ctx->a_split[1]);
     cudaFree(ctx->tc_ws);
     cudaFree(ctx->mg_ws);
+    cudaFree(ctx->mg_tc);
     cudaFree(ctx->tc_counters);
     cudaFree(ctx->stage);
     if (ctx->prof) {

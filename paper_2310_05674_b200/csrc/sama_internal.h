@@ -91,6 +91,8 @@ struct sama_ctx {
     int* tc_counters;              // device [kTcCounters], zero between launches
     float* mg_ws;                  // device: workspace of the direct gradient (activations, dz, losses)
     size_t mg_ws_floats;
+    float* mg_tc;                  // device: TF32 operand buffers of the direct gradient's tensor-core path
+    size_t mg_tc_floats;
     float* stage;                  // device: staging of the host entry point (allocated on first use)
     size_t stage_bytes;
     sama::Profiler* prof;          // host
@@ -233,6 +235,8 @@ cudaError_t launch_head_ce_fd(sama_ctx* ctx, const float* h_plus, const float* h
 
 // meta_grad.cu : direct gradient dL_meta/dtheta (Eq. 1)
 size_t meta_grad_workspace_floats(const sama_mlp_t* mlp, int64_t B);
+size_t meta_grad_tc_floats(const sama_mlp_t* mlp, int64_t B);
+SplitLayout make_split_layout(const sama_mlp_t* mlp);  // sama_api.cu
 cudaError_t run_meta_grad(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta, const float* X, const int32_t* y,
                           int32_t B, float* g_out, float* loss_out, cudaStream_t st);
 

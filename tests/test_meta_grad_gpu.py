@@ -1,7 +1,7 @@
 """GPU parity of the direct gradient dL_meta/dtheta (Eq. 1) against the CPU checker.
 
-Inputs are conditioned so that no hidden pre-activation lies within 1e-3 of the ReLU kink (see
-away_from_kinks).  Tolerance: every entry within 5e-5 of the largest magnitude in its own layer block
+Inputs are conditioned so that no hidden pre-activation lies within max(1e-3, 1e-4 max|z|) of the
+ReLU kink (see away_from_kinks).  Tolerance: every entry within 5e-5 of the largest magnitude in its own layer block
 (weights or biases): three chained fp32 contractions of length up to K = 4096, each with about
 sqrt(K) 2^-24 = 4e-6 of relative rounding, times a margin of 4.  Each entry is an fp32 sum of B products (and the dz it is built from went through the
 fp32 forward pass), so its error scales with the block's magnitude, not with the entry's own."""
@@ -28,10 +28,11 @@ def blocks(dims):
     return out
 
 
-def away_from_kinks(dims, theta, X, tau=1e-3):
-    """Deterministically nudges hidden-layer biases until no hidden pre-activation lies within tau of
-    zero.  At a ReLU kink the derivative is not determined within fp32 rounding of the forward pass
-    (both 0 and 1 are right), so a well-posed comparison needs inputs that stay clear of it."""
+def away_from_kinks(dims, theta, X, tau_abs=1e-3, tau_rel=1e-4):
+    """Deterministically nudges hidden-layer biases until no hidden pre-activation lies within
+    tau = max(tau_abs, tau_rel * max|z|) of zero.  At a ReLU kink the derivative is not determined
+    within the rounding of the forward pass (both 0 and 1 are right; the rounding scales with the
+    size of the pre-activations), so a well-posed comparison needs inputs that stay clear of it."""
     theta = theta.copy()
     L = len(dims) - 1
     h = X.astype(np.float64)
@@ -41,6 +42,7 @@ def away_from_kinks(dims, theta, X, tau=1e-3):
         Wl = theta[o:o + nw].astype(np.float64).reshape(dims[l + 1], dims[l])
         bias = theta[o + nw:o + nw + dims[l + 1]]
         zw = h @ Wl.T
+        tau = max(tau_abs, tau_rel * float(np.abs(zw).max()))
         for it in range(50):
             z = zw + bias.astype(np.float64)
             bad = np.unique(np.argwhere(np.abs(z) < tau)[:, 1])
@@ -54,13 +56,13 @@ def away_from_kinks(dims, theta, X, tau=1e-3):
     return theta
 
 
-def check(dims, batch, seed, clean=True):
+def check(dims, batch, seed, clean=True, gemm_mode=0):
     cfg, w = W.custom_mlp(dims, batch, seed=seed)
     theta = (w["theta"] + 0.05 * W.normal(seed, 99, cfg.n_params).astype(np.float32)).astype(np.float32)
     theta = away_from_kinks(dims, theta, w["X"])
     y = w["y_clean"] if clean else w["y"]
     loss_ref, g_ref = oracle.meta_grad(dims, theta, w["X"], y)
-    with Ctx(cfg.n_params, batch, dims) as ctx:
+    with Ctx(cfg.n_params, batch, dims, gemm_mode) as ctx:
         g = torch.full((cfg.n_params,), float("nan"), dtype=torch.float32, device=DEV)
         loss = torch.zeros(1, dtype=torch.float32, device=DEV)
         th, X, yd = dev(theta), dev(w["X"]), dev(y)
@@ -71,7 +73,9 @@ def check(dims, batch, seed, clean=True):
         torch.cuda.synchronize()
         assert np.array_equal(g.cpu().numpy(), g1)          # bitwise reproducible
         assert B.sama_device_status(ctx.h) == 0
-    assert float(loss.item()) == pytest.approx(loss_ref, rel=2e-6)
+    # the mean loss is a by-product; with the weight noise added above the logits reach ~100, so fp32 / 3xTF32
+    # rounding of the logits (2^-22 of the summed magnitudes) shows up at a few 1e-5 of the loss
+    assert float(loss.item()) == pytest.approx(loss_ref, rel=1e-4)
     worst = 0.0
     for a, b in blocks(dims):
         scale = np.abs(g_ref[a:b]).max()
@@ -79,28 +83,34 @@ def check(dims, batch, seed, clean=True):
             assert np.all(g1[a:b] == 0)
             continue
         worst = max(worst, float(np.abs(g1[a:b] - g_ref[a:b]).max() / scale))
-    print("\n[meta_grad] dims=%s B=%d: worst block-relative error %.2e" % (dims, batch, worst))
-    assert worst <= 5e-5, worst
+    print("\n[meta_grad] dims=%s B=%d gemm_mode=%d: worst block-relative error %.2e" % (dims, batch, gemm_mode, worst))
+    # tensor-core accumulators round toward zero: 3 K / 8 accumulations of up to 2^-24 (mean) each
+    tol = 5e-5 + (4 * 3 * max(dims) / 8 * 2.0 ** -24 if gemm_mode == 2 else 0.0)
+    assert worst <= tol, worst
     return theta, w, g1, g_ref
 
 
 @pytest.mark.parametrize("dims,batch", [((12, 5), 1), ((33, 17, 12, 6), 7), ((100, 50, 3), 129), ((257, 130, 66, 11), 65),
                                         ((40, 200, 72, 24), 257)])
-def test_meta_grad_parity_ragged(dims, batch):
-    check(dims, batch, seed=sum(dims))
+@pytest.mark.parametrize("gemm_mode", [1, 2])
+def test_meta_grad_parity_ragged(dims, batch, gemm_mode):
+    check(dims, batch, seed=sum(dims), gemm_mode=gemm_mode)
 
 
-def test_meta_grad_parity_tiny_and_mlp3072():
-    check(W.CONFIGS["tiny"].dims, W.CONFIGS["tiny"].batch, 0)
-    check(W.CONFIGS["mlp3072"].dims, W.CONFIGS["mlp3072"].batch, 0, clean=False)
+@pytest.mark.parametrize("gemm_mode", [1, 2])
+def test_meta_grad_parity_tiny_and_mlp3072(gemm_mode):
+    check(W.CONFIGS["tiny"].dims, W.CONFIGS["tiny"].batch, 0, gemm_mode=gemm_mode)
+    check(W.CONFIGS["mlp3072"].dims, W.CONFIGS["mlp3072"].batch, 0, clean=False, gemm_mode=gemm_mode)
 
 
-def test_meta_grad_parity_head1024():
-    check(W.CONFIGS["head1024"].dims, 1024, 0)
+@pytest.mark.parametrize("gemm_mode", [1, 2])
+def test_meta_grad_parity_head1024(gemm_mode):
+    check(W.CONFIGS["head1024"].dims, 1024, 0, gemm_mode=gemm_mode)
 
 
-def test_meta_grad_parity_wide_dims_small_batch():
-    check(W.CONFIGS["wide4096"].dims, 48, 0)
+@pytest.mark.parametrize("gemm_mode", [1, 2])
+def test_meta_grad_parity_wide_dims_small_batch(gemm_mode):
+    check(W.CONFIGS["wide4096"].dims, 48, 0, gemm_mode=gemm_mode)
 
 
 def test_meta_grad_feeds_the_step():
