@@ -9,18 +9,22 @@
 // forward passes by 2 eps_fd, which amplifies rounding by 1/eps_fd; plain TF32
 // (2^-11) would drown the signal, which is why the split is needed.
 //
-// Structure of gemm_tf32x3_kernel (one 128 x BN output tile per CTA, 192 threads):
+// Structure of gemm_tf32x3_kernel (one 128 x BN output tile per CTA, or one 256 x BN tile per CTA
+// pair; 2 + 4 or 2 + 8 warps):
 //   warp 0    : TMA producer.  Per k-block of 32 floats it loads four tiles
 //               (A hi/lo: 128 x 32, W hi/lo: BN x 32) with cp.async.bulk.tensor
 //               into 128-byte-swizzled shared memory and signals a "full"
 //               mbarrier with the byte count.  No multicast.
-//   warp 1    : allocates tensor memory, then one lane issues, per k-block,
-//               4 k-steps x 3 tcgen05.mma kind::tf32 (M = 128, N = BN, K = 8)
-//               from shared-memory descriptors and commits to the stage's
-//               "empty" mbarrier; a last commit signals the accumulator.
-//   warps 2-5 : epilogue.  Each warp reads its 32 lanes of the accumulator with
-//               tcgen05.ld, adds the bias, applies ReLU, and either stores fp32
-//               logits or stores the next layer's hi/lo operands directly.
+//   warp 1    : allocates tensor memory (two accumulators), then one lane issues,
+//               per k-block, 4 k-steps x 3 tcgen05.mma kind::tf32 (M = 128 or 256,
+//               N = BN, K = 8) from shared-memory descriptors and commits to the
+//               stage's "empty" mbarrier; every few k-blocks it commits the chunk's
+//               accumulator and moves to the other one.
+//   warps 2.. : epilogue.  Each warp reads its 32 lanes of a finished chunk with
+//               tcgen05.ld and adds it to a running fp32 sum in registers (the
+//               tensor core's own accumulation rounds toward zero, see kChunkKb);
+//               after the last chunk it adds the bias, applies ReLU, and either
+//               stores fp32 results or the next layer's hi/lo operands directly.
 // Operands are K-major in global memory ([rows][K], K padded to a multiple of
 // 32 with zeros), which is what both TMA and the K-major UMMA descriptor want.
 // Every mbarrier wait is bounded: if one expires the CTA raises
@@ -39,7 +43,13 @@ namespace {
 constexpr int BM = 128;       // rows of the output tile = TMEM lanes
 constexpr int BKF = 32;       // floats per k-block = one 128-byte swizzle row
 constexpr int UMMA_K = 8;     // K of one kind::tf32 instruction
-constexpr int kThreads = 192;
+// The tensor core adds each product into its fp32 accumulator with round-toward-zero, so a long
+// contraction kept in tensor memory drifts towards zero by about 2^-24 per instruction (measured:
+// 6e-5 relative at K = 4096).  The contraction is therefore cut into chunks of kChunkKb k-blocks that
+// alternate between two accumulators in tensor memory; the epilogue warps add each finished chunk
+// into fp32 registers (round-to-nearest) while the next chunk is being multiplied.
+constexpr int kChunkKb = 4;
+__host__ __device__ constexpr int threads_for(int epi) { return 64 + 32 * epi; }  // epi = 4 or 8 epilogue warps
 constexpr long long kWaitCycles = 4000000000LL;  // ~2 s at 2 GHz
 
 // `wrows` = rows of W one CTA stages per k-block: BN, or BN / 2 when a CTA pair shares the W tile.
@@ -150,16 +160,30 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
-    uint32_t r[16];
+// Two 16-column reads in flight, one wait.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+    uint32_t r[32];
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr));
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr + 16u));
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Arrival on a barrier that may live in the other CTA of the pair (shared::cluster address).
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
 // Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes
@@ -196,6 +220,7 @@ struct TcArgs {
     const float* mask;     // [M][ldm] or null: results are zeroed where mask <= 0
     int ldm;
     int tiles_m, tiles_n, group_n;
+    int chunk_kb;              // k-blocks per accumulator chunk
     int splits, kb_per_split;  // split-K: grid.z = 2 * splits, each CTA takes kb_per_split k-blocks
     float* ws;                 // split-K partial tiles [2 * tiles][splits][BM][BN]
     int* counters;             // split-K arrival counters [2 * tiles], zero between launches
@@ -206,8 +231,8 @@ struct TcArgs {
 // PAIR = true: two CTAs of a cluster work on one 256 x BN tile.  Each stages its own 128 rows of A and half of
 // the W tile; the leader CTA issues cta_group::2 products that read both CTAs' shared memory and write both
 // CTAs' tensor memory.  Per CTA and flop that is fewer operand bytes than two independent 128 x BN tiles.
-template <int BN, bool PAIR>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int BN, bool PAIR, int EPI>
+__global__ void __launch_bounds__(threads_for(EPI), 1)
 gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
                    const __grid_constant__ CUtensorMap map_w_hi, const __grid_constant__ CUtensorMap map_w_lo,
                    TcArgs args) {
@@ -215,7 +240,11 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     constexpr int STAGES = stages_for(WROWS);
     constexpr int A_BYTES = BM * BKF * 4, W_BYTES = WROWS * BKF * 4;
     constexpr int STAGE = stage_bytes(WROWS);
-    constexpr uint32_t TMEM_COLS = BN < 32 ? 32 : BN;
+    constexpr uint32_t ACC_COLS = BN < 32 ? 32 : BN;   // one accumulator
+    constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;       // two, alternating by chunk
+    constexpr int CPW = BN / (EPI / 4);                // accumulator columns per epilogue thread
+    constexpr int ACC_REGS = CPW < 32 ? 32 : CPW;
+    static_assert(CPW <= 128, "at most 128 accumulator columns per epilogue thread");
     constexpr uint32_t IDESC = make_idesc(BN, PAIR ? 2 * BM : BM);
 
     extern __shared__ uint8_t smem_raw[];
@@ -223,8 +252,9 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     const uint32_t bars = base + STAGES * STAGE;                   // full[STAGES], empty[STAGES], accum, tmem slot
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
-    const uint32_t accum_bar = bars + 8u * (2 * STAGES);
-    const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 1);
+    auto acc_full_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };        // chunk in accumulator b is complete
+    auto acc_empty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };   // accumulator b has been read out
+    const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 4);
     const uint32_t abort_slot = tmem_slot + 4;
     volatile uint32_t* abort_flag =
         reinterpret_cast<volatile uint32_t*>(smem_raw + (abort_slot - smem_u32(smem_raw)));
@@ -261,7 +291,10 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
             mbar_init(full_bar(s), 1);
             mbar_init(empty_bar(s), 1);
         }
-        mbar_init(accum_bar, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(acc_full_bar(b), 1);
+            mbar_init(acc_empty_bar(b), EPI * (PAIR ? 2 : 1));  // one arrival per epilogue warp (of both CTAs of a pair)
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -324,54 +357,93 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
             bool ok = true;
             for (int kb = 0; kb < num_kb && ok; ++kb) {
                 const int s = kb % STAGES;
+                const int chunk = kb / args.chunk_kb, buf = chunk & 1;
+                const bool chunk_first = (kb - chunk * args.chunk_kb) == 0;
+                if (chunk_first && chunk >= 2) {
+                    // the epilogue warps have drained this accumulator's previous chunk
+                    if (!mbar_wait(acc_empty_bar(buf), ((chunk >> 1) - 1) & 1)) { raise_timeout(); ok = false; break; }
+                }
                 if (!mbar_wait(full_bar(s), (kb / STAGES) & 1)) { raise_timeout(); ok = false; break; }
                 if (*abort_flag) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t st = base + s * STAGE;
+                const uint32_t acc = tmem_base + (uint32_t)buf * ACC_COLS;
                 const uint64_t a_hi = make_desc(st), a_lo = make_desc(st + A_BYTES);
                 const uint64_t w_hi = make_desc(st + 2 * A_BYTES), w_lo = make_desc(st + 2 * A_BYTES + W_BYTES);
 #pragma unroll
                 for (int k = 0; k < BKF / UMMA_K; ++k) {
                     const uint64_t adv = (uint64_t)((k * UMMA_K * 4) >> 4);  // 32 bytes per k-step inside the swizzled row
+                    const uint32_t keep = (chunk_first && k == 0) ? 0u : 1u;  // a chunk starts from zero
                     if (PAIR) {
-                        umma_tf32_pair(tmem_base, a_hi + adv, w_lo + adv, IDESC, (kb | k) != 0);
-                        umma_tf32_pair(tmem_base, a_lo + adv, w_hi + adv, IDESC, 1);
-                        umma_tf32_pair(tmem_base, a_hi + adv, w_hi + adv, IDESC, 1);
+                        umma_tf32_pair(acc, a_hi + adv, w_lo + adv, IDESC, keep);
+                        umma_tf32_pair(acc, a_lo + adv, w_hi + adv, IDESC, 1);
+                        umma_tf32_pair(acc, a_hi + adv, w_hi + adv, IDESC, 1);
                     } else {
-                        umma_tf32(tmem_base, a_hi + adv, w_lo + adv, IDESC, (kb | k) != 0);
-                        umma_tf32(tmem_base, a_lo + adv, w_hi + adv, IDESC, 1);
-                        umma_tf32(tmem_base, a_hi + adv, w_hi + adv, IDESC, 1);
+                        umma_tf32(acc, a_hi + adv, w_lo + adv, IDESC, keep);
+                        umma_tf32(acc, a_lo + adv, w_hi + adv, IDESC, 1);
+                        umma_tf32(acc, a_hi + adv, w_hi + adv, IDESC, 1);
                     }
                 }
                 // frees the stage (in both CTAs of a pair) once these products have read it
                 if (PAIR) umma_commit_pair(empty_bar(s)); else umma_commit(empty_bar(s));
+                if (kb - chunk * args.chunk_kb == args.chunk_kb - 1 || kb == num_kb - 1) {
+                    if (PAIR) umma_commit_pair(acc_full_bar(buf)); else umma_commit(acc_full_bar(buf));
+                }
             }
-            if (ok) { if (PAIR) umma_commit_pair(accum_bar); else umma_commit(accum_bar); }
         }
     } else {
         // -------------------------------------------------------------- epilogue
-        const int q = warp & 3;  // a warp may only touch TMEM lanes [32 q, 32 q + 32)
+        const int q = warp & 3;            // a warp may only touch TMEM lanes [32 q, 32 q + 32)
+        const int col0 = ((warp - 2) >> 2) * CPW;  // with eight epilogue warps, two share a lane quarter and split the columns
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)col0;
+        float acc[ACC_REGS];
+#pragma unroll
+        for (int j = 0; j < ACC_REGS; ++j) acc[j] = 0.f;
         bool ok = true;
-        if (lane == 0) {
-            // the accumulator is final when its barrier flips, or never if a producer gave up
-            const long long t0 = clock64();
-            while (!mbar_try(accum_bar, 0)) {
-                if (*abort_flag) { ok = false; break; }
-                if (clock64() - t0 > 2 * kWaitCycles) { raise_timeout(); ok = false; break; }
+        const int n_chunks = (num_kb + args.chunk_kb - 1) / args.chunk_kb;
+#pragma unroll 1
+        for (int chunk = 0; chunk < n_chunks; ++chunk) {
+            const int buf = chunk & 1;
+            if (lane == 0) {
+                // the chunk is complete when its barrier flips, or never if a producer gave up
+                const long long t0 = clock64();
+                while (!mbar_try(acc_full_bar(buf), (chunk >> 1) & 1)) {
+                    if (*abort_flag) { ok = false; break; }
+                    if (clock64() - t0 > 2 * kWaitCycles) { raise_timeout(); ok = false; break; }
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t src = lane_addr + (uint32_t)buf * ACC_COLS;
+#pragma unroll
+            for (int c = 0; c < ACC_REGS; c += 32) {
+                float v[32];
+                tmem_ld32(src + c, v);   // all lanes take part (sync.aligned)
+#pragma unroll
+                for (int j = 0; j < 32; ++j) acc[c + j] += v[j];
+            }
+            // this warp's reads are done: hand the accumulator back to the MMA issuer
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0 && chunk + 2 < n_chunks) {
+                if (PAIR) mbar_arrive_cluster(acc_empty_bar(buf) & kPeerBitMask); else mbar_arrive(acc_empty_bar(buf));
             }
         }
-        ok = __shfl_sync(0xffffffffu, ok, 0);
-        // the four epilogue warps proceed together or not at all (they meet again at named barrier 1)
+        // the epilogue warps proceed together or not at all (they meet again at named barrier 1)
         volatile uint32_t* ok_slots = last_flag + 1;
-        if (lane == 0) ok_slots[q] = ok ? 1u : 0u;
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        ok = (ok_slots[0] & ok_slots[1] & ok_slots[2] & ok_slots[3]) != 0;
+        if (lane == 0) ok_slots[warp - 2] = ok ? 1u : 0u;
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * EPI) : "memory");
+        {
+            uint32_t all = 1u;
+#pragma unroll
+            for (int w = 0; w < EPI; ++w) all &= ok_slots[w];
+            ok = all != 0;
+        }
         if (ok) {
-            tc_fence_after();
             const int row = q * 32 + lane;
             const int m = m0 + row;
             const float* bias = br ? args.bias[1] : args.bias[0];
-            const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
             // Split-K: every CTA of a tile stores its raw partial; the last one to arrive adds the
             // partials in split order (so the sum does not depend on which CTA that is) and finishes.
             const float* part = nullptr;
@@ -379,89 +451,86 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
             if (args.splits > 1) {
                 const int tile_lin = br * (args.tiles_m * args.tiles_n) + (int)blockIdx.x;
                 float* base_ws = args.ws + (int64_t)tile_lin * args.splits * (BM * BN);
-                float* mine = base_ws + ((int64_t)split * BM + row) * BN;
-#pragma unroll 1
-                for (int c = 0; c < BN; c += 16) {
-                    float v[16];
-                    tmem_ld16(lane_addr + c, v);
+                float* mine = base_ws + ((int64_t)split * BM + row) * BN + col0;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        __stcg(reinterpret_cast<float4*>(mine + c) + j,
-                               make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]));
-                }
+                for (int c = 0; c < CPW; c += 4)
+                    __stcg(reinterpret_cast<float4*>(mine + c), make_float4(acc[c], acc[c + 1], acc[c + 2], acc[c + 3]));
                 __threadfence();
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                asm volatile("bar.sync 1, %0;" ::"n"(32 * EPI) : "memory");
                 if (warp == 2 && lane == 0) {
                     const int prev = atomicAdd(args.counters + tile_lin, 1);
                     const bool is_last = (prev == args.splits - 1);
                     if (is_last) args.counters[tile_lin] = 0;  // every CTA of the tile has arrived
                     *last_flag = is_last ? 1u : 0u;
                 }
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                asm volatile("bar.sync 1, %0;" ::"n"(32 * EPI) : "memory");
                 finish = (*last_flag != 0);
                 if (finish) __threadfence();
-                part = base_ws + (int64_t)row * BN;
+                part = base_ws + (int64_t)row * BN + col0;
             }
-#pragma unroll 1
-            for (int c = 0; finish && c < BN; c += 16) {
-                float v[16];
-                if (part) {
+            if (finish) {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] = 0.f;
-                    for (int sp = 0; sp < args.splits; ++sp) {
-                        const float4* src = reinterpret_cast<const float4*>(part + (int64_t)sp * (BM * BN) + c);
+                for (int c = 0; c < CPW; c += 16) {
+                    float v[16];
+                    if (part) {
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const float4 t = __ldcg(src + j);
-                            v[4 * j] += t.x; v[4 * j + 1] += t.y; v[4 * j + 2] += t.z; v[4 * j + 3] += t.w;
+                        for (int j = 0; j < 16; ++j) v[j] = 0.f;
+                        for (int sp = 0; sp < args.splits; ++sp) {
+                            const float4* src = reinterpret_cast<const float4*>(part + (int64_t)sp * (BM * BN) + c);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const float4 t = __ldcg(src + j);
+                                v[4 * j] += t.x; v[4 * j + 1] += t.y; v[4 * j + 2] += t.z; v[4 * j + 3] += t.w;
+                            }
                         }
-                    }
-                } else {
-                    tmem_ld16(lane_addr + c, v);   // all lanes take part (sync.aligned)
-                }
-                const int n = n0 + c;
-                if (m < args.M) {
+                    } else {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        float x = v[j] + ((bias != nullptr && n + j < args.N) ? bias[n + j] : 0.f);
-                        if (args.relu && x < 0.f) x = 0.f;
-                        v[j] = x;
+                        for (int j = 0; j < 16; ++j) v[j] = acc[c + j];
                     }
-                    if (args.mask) {  // backward pass: the derivative passes only where the forward activation was positive
-                        const float* mk = args.mask + (int64_t)m * args.ldm + n;
-#pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (n + j < args.N && !(mk[j] > 0.f)) v[j] = 0.f;
-                    }
-                    if (args.last || args.both) {
-                        float* dst = (br ? args.out_f32[1] : args.out_f32[0]) + (int64_t)m * args.ldc + n;
-                        if (n + 15 < args.N && (args.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
-#pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                reinterpret_cast<float4*>(dst)[j] =
-                                    make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                if (n + j < args.N) dst[j] = v[j];
-                        }
-                    }
-                    if (!args.last && n < args.ld_next) {
-                        // columns in [N, ld_next) are the next layer's zero padding along K
-                        const int64_t off = ((int64_t)br * args.M + m) * args.ld_next + n;
-                        float hi[16], lo[16];
+                    const int n = n0 + col0 + c;
+                    if (m < args.M) {
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
-                            const float x = (n + j < args.N) ? v[j] : 0.f;
-                            hi[j] = to_tf32(x);
-                            lo[j] = to_tf32(x - hi[j]);
+                            float x = v[j] + ((bias != nullptr && n + j < args.N) ? bias[n + j] : 0.f);
+                            if (args.relu && x < 0.f) x = 0.f;
+                            v[j] = x;
                         }
-                        float4* dh = reinterpret_cast<float4*>(args.out_hi + off);
-                        float4* dl = reinterpret_cast<float4*>(args.out_lo + off);
+                        if (args.mask) {  // backward pass: the derivative passes only where the forward activation was positive
+                            const float* mk = args.mask + (int64_t)m * args.ldm + n;
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            dh[j] = make_float4(hi[4 * j], hi[4 * j + 1], hi[4 * j + 2], hi[4 * j + 3]);
-                            dl[j] = make_float4(lo[4 * j], lo[4 * j + 1], lo[4 * j + 2], lo[4 * j + 3]);
+                            for (int j = 0; j < 16; ++j)
+                                if (n + j < args.N && !(mk[j] > 0.f)) v[j] = 0.f;
+                        }
+                        if (args.last || args.both) {
+                            float* dst = (br ? args.out_f32[1] : args.out_f32[0]) + (int64_t)m * args.ldc + n;
+                            if (n + 15 < args.N && (args.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+#pragma unroll
+                                for (int j = 0; j < 4; ++j)
+                                    reinterpret_cast<float4*>(dst)[j] =
+                                        make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 16; ++j)
+                                    if (n + j < args.N) dst[j] = v[j];
+                            }
+                        }
+                        if (!args.last && n < args.ld_next) {
+                            // columns in [N, ld_next) are the next layer's zero padding along K
+                            const int64_t off = ((int64_t)br * args.M + m) * args.ld_next + n;
+                            float hi[16], lo[16];
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const float x = (n + j < args.N) ? v[j] : 0.f;
+                                hi[j] = to_tf32(x);
+                                lo[j] = to_tf32(x - hi[j]);
+                            }
+                            float4* dh = reinterpret_cast<float4*>(args.out_hi + off);
+                            float4* dl = reinterpret_cast<float4*>(args.out_lo + off);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                dh[j] = make_float4(hi[4 * j], hi[4 * j + 1], hi[4 * j + 2], hi[4 * j + 3]);
+                                dl[j] = make_float4(lo[4 * j], lo[4 * j + 1], lo[4 * j + 2], lo[4 * j + 3]);
+                            }
                         }
                     }
                 }
@@ -590,17 +659,17 @@ bool make_map(CUtensorMap* map, const float* base, int ld, int64_t rows, int sla
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, bool PAIR>
+template <int BN, bool PAIR, int EPI>
 cudaError_t launch_tc(const CUtensorMap maps[4], const TcArgs& a, dim3 grid, cudaStream_t st) {
     constexpr int kSmem = smem_bytes(PAIR ? BN / 2 : BN);
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tf32x3_kernel<BN, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemm_tf32x3_kernel<BN, PAIR, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kSmem);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    return launch_clustered(PAIR ? 2 : 1, gemm_tf32x3_kernel<BN, PAIR>, grid, dim3(kThreads), (size_t)kSmem, st,
+    return launch_clustered(PAIR ? 2 : 1, gemm_tf32x3_kernel<BN, PAIR, EPI>, grid, dim3(threads_for(EPI)), (size_t)kSmem, st,
                             maps[0], maps[1], maps[2], maps[3], a);
 }
 
@@ -727,14 +796,17 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     if (const char* e = std::getenv("SAMA_TC_GROUP")) { const int g = std::atoi(e); if (g >= 1 && g <= a.tiles_n) a.group_n = g; }
     dim3 grid(a.tiles_m * a.tiles_n * (pair ? 2 : 1), 1, nbr * a.splits);
     KernelScope scope(ctx, SAMA_K_GEMM_TF32X3, L.layer, st);
+    a.chunk_kb = kChunkKb;
+    if (const char* e = std::getenv("SAMA_TC_CHUNK")) { const int c = std::atoi(e); if (c >= 1) a.chunk_kb = c; }
+    // eight epilogue warps (two per lane quarter, each taking half of the columns) except on the 16-wide tile
     if (pair) {
-        if (bn == 64) return launch_tc<64, true>(maps, a, grid, st);
-        if (bn == 256) return launch_tc<256, true>(maps, a, grid, st);
-        return launch_tc<128, true>(maps, a, grid, st);
+        if (bn == 64) return launch_tc<64, true, 8>(maps, a, grid, st);
+        if (bn == 256) return launch_tc<256, true, 8>(maps, a, grid, st);
+        return launch_tc<128, true, 8>(maps, a, grid, st);
     }
-    if (bn == 16) return launch_tc<16, false>(maps, a, grid, st);
-    if (bn == 64) return launch_tc<64, false>(maps, a, grid, st);
-    return launch_tc<128, false>(maps, a, grid, st);
+    if (bn == 16) return launch_tc<16, false, 4>(maps, a, grid, st);
+    if (bn == 64) return launch_tc<64, false, 8>(maps, a, grid, st);
+    return launch_tc<128, false, 8>(maps, a, grid, st);
 }
 
 }  // namespace sama

@@ -1,10 +1,12 @@
 """GPU parity of the direct gradient dL_meta/dtheta (Eq. 1) against the CPU checker.
 
 Inputs are conditioned so that no hidden pre-activation lies within max(1e-3, 1e-4 max|z|) of the
-ReLU kink (see away_from_kinks).  Tolerance: every entry within 5e-5 of the largest magnitude in its own layer block
-(weights or biases): three chained fp32 contractions of length up to K = 4096, each with about
-sqrt(K) 2^-24 = 4e-6 of relative rounding, times a margin of 4.  Each entry is an fp32 sum of B products (and the dz it is built from went through the
-fp32 forward pass), so its error scales with the block's magnitude, not with the entry's own."""
+ReLU kink (see away_from_kinks).  Tolerance: every entry within 5e-5 of the largest magnitude in its
+own layer block (weights or biases): three chained fp32 contractions of length up to K = 4096, each
+with about sqrt(K) 2^-24 = 4e-6 of relative rounding, times a margin of 4.  Each entry is an fp32 sum
+of B products (and the dz it is built from went through the fp32 forward pass), so its error scales
+with the block's magnitude, not with the entry's own.  Both GEMM modes (fp32 FMA and the three-product
+TF32 tensor-core path) are held to the same bound."""
 import numpy as np
 import pytest
 import torch
@@ -73,9 +75,10 @@ def check(dims, batch, seed, clean=True, gemm_mode=0):
         torch.cuda.synchronize()
         assert np.array_equal(g.cpu().numpy(), g1)          # bitwise reproducible
         assert B.sama_device_status(ctx.h) == 0
-    # the mean loss is a by-product; with the weight noise added above the logits reach ~100, so fp32 / 3xTF32
-    # rounding of the logits (2^-22 of the summed magnitudes) shows up at a few 1e-5 of the loss
-    assert float(loss.item()) == pytest.approx(loss_ref, rel=1e-4)
+    # the mean loss is a by-product; with the weight noise added above the logits reach ~100, so fp32 rounding of
+    # the logits (sqrt(K) 2^-24 of their magnitude) shows up at a few 1e-6 of the loss.  A tensor-core
+    # accumulator left to drift over the whole contraction (it rounds toward zero) would miss this by 4x.
+    assert float(loss.item()) == pytest.approx(loss_ref, rel=2e-5)
     worst = 0.0
     for a, b in blocks(dims):
         scale = np.abs(g_ref[a:b]).max()
@@ -84,9 +87,7 @@ def check(dims, batch, seed, clean=True, gemm_mode=0):
             continue
         worst = max(worst, float(np.abs(g1[a:b] - g_ref[a:b]).max() / scale))
     print("\n[meta_grad] dims=%s B=%d gemm_mode=%d: worst block-relative error %.2e" % (dims, batch, gemm_mode, worst))
-    # tensor-core accumulators round toward zero: 3 K / 8 accumulations of up to 2^-24 (mean) each
-    tol = 5e-5 + (4 * 3 * max(dims) / 8 * 2.0 ** -24 if gemm_mode == 2 else 0.0)
-    assert worst <= tol, worst
+    assert worst <= 5e-5, worst
     return theta, w, g1, g_ref
 
 
