@@ -78,14 +78,16 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: false if the phase did not complete within kWaitCycles.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait: false if the phase did not complete within kWaitCycles, or if another role of the CTA
+// has given up meanwhile (`abort`, looked at only once the first try has failed).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile uint32_t* abort = nullptr) {
     if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 256; ++i)
             if (mbar_try(bar, parity)) return true;
+        if (abort && *abort) return false;
         if (clock64() - t0 > kWaitCycles) return false;
     }
 }
@@ -220,7 +222,6 @@ struct TcArgs {
     const float* mask;     // [M][ldm] or null: results are zeroed where mask <= 0
     int ldm;
     int tiles_m, tiles_n, group_n;
-    int chunk_kb;              // k-blocks per accumulator chunk
     int splits, kb_per_split;  // split-K: grid.z = 2 * splits, each CTA takes kb_per_split k-blocks
     float* ws;                 // split-K partial tiles [2 * tiles][splits][BM][BN]
     int* counters;             // split-K arrival counters [2 * tiles], zero between launches
@@ -240,12 +241,18 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     constexpr int STAGES = stages_for(WROWS);
     constexpr int A_BYTES = BM * BKF * 4, W_BYTES = WROWS * BKF * 4;
     constexpr int STAGE = stage_bytes(WROWS);
-    constexpr uint32_t ACC_COLS = BN < 32 ? 32 : BN;   // one accumulator
+    // Single-CTA tiles of 64 or 128 columns issue two products per k-step instead of three: W hi and W lo
+    // sit back to back in shared memory, so A hi x [W hi; W lo]^T is one instruction of twice the width
+    // (A hi is fetched once, and fewer, larger instructions keep the tensor pipe fuller), and A lo x W hi^T
+    // joins the small terms in the second half of the accumulator.  The epilogue adds the two halves.
+    constexpr bool CONCAT = !PAIR && BN >= 64;
+    constexpr uint32_t ACC_COLS = CONCAT ? 2 * BN : (BN < 32 ? 32 : BN);   // one accumulator
     constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;       // two, alternating by chunk
     constexpr int CPW = BN / (EPI / 4);                // accumulator columns per epilogue thread
     constexpr int ACC_REGS = CPW < 32 ? 32 : CPW;
     static_assert(CPW <= 128, "at most 128 accumulator columns per epilogue thread");
     constexpr uint32_t IDESC = make_idesc(BN, PAIR ? 2 * BM : BM);
+    constexpr uint32_t IDESC_CAT = make_idesc(CONCAT ? 2 * BN : BN, BM);
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // tiles need 1024-byte alignment
@@ -321,11 +328,10 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         if (lane == 0) {
             int issued = 0;
             const int za = args.shared_a ? 0 : br;
+            int s = 0;
+            uint32_t empty_parity = 1;  // parity of the phase that frees stage s for its next round
             for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t round = kb / STAGES;
-                if (kb >= STAGES && !mbar_wait(empty_bar(s), (round - 1) & 1)) { raise_timeout(); break; }
-                if (*abort_flag) break;
+                if (kb >= STAGES && !mbar_wait(empty_bar(s), empty_parity, abort_flag)) { raise_timeout(); break; }
                 const uint32_t st = base + s * STAGE;
                 const int kx = (kb_begin + kb) * BKF;
                 if (PAIR) {
@@ -344,6 +350,7 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                     tma_load_3d(st + 2 * A_BYTES + W_BYTES, &map_w_lo, full_bar(s), kx, n0, br);
                 }
                 issued = kb + 1;
+                if (++s == STAGES) { s = 0; empty_parity ^= 1u; }
             }
             if (*abort_flag && rank == 0) {
                 // let the copies already issued land before the CTA's shared memory goes away
@@ -355,16 +362,16 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         // ------------------------------------------------------------ MMA issuer (the leader's, for a pair)
         if (lane == 0 && rank == 0) {
             bool ok = true;
+            int s = 0, in_chunk = 0, chunk = 0;
+            uint32_t full_parity = 0;
             for (int kb = 0; kb < num_kb && ok; ++kb) {
-                const int s = kb % STAGES;
-                const int chunk = kb / args.chunk_kb, buf = chunk & 1;
-                const bool chunk_first = (kb - chunk * args.chunk_kb) == 0;
+                const int buf = chunk & 1;
+                const bool chunk_first = in_chunk == 0;
                 if (chunk_first && chunk >= 2) {
                     // the epilogue warps have drained this accumulator's previous chunk
-                    if (!mbar_wait(acc_empty_bar(buf), ((chunk >> 1) - 1) & 1)) { raise_timeout(); ok = false; break; }
+                    if (!mbar_wait(acc_empty_bar(buf), ((chunk >> 1) - 1) & 1, abort_flag)) { raise_timeout(); ok = false; break; }
                 }
-                if (!mbar_wait(full_bar(s), (kb / STAGES) & 1)) { raise_timeout(); ok = false; break; }
-                if (*abort_flag) { ok = false; break; }
+                if (!mbar_wait(full_bar(s), full_parity, abort_flag)) { raise_timeout(); ok = false; break; }
                 tc_fence_after();
                 const uint32_t st = base + s * STAGE;
                 const uint32_t acc = tmem_base + (uint32_t)buf * ACC_COLS;
@@ -378,6 +385,9 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                         umma_tf32_pair(acc, a_hi + adv, w_lo + adv, IDESC, keep);
                         umma_tf32_pair(acc, a_lo + adv, w_hi + adv, IDESC, 1);
                         umma_tf32_pair(acc, a_hi + adv, w_hi + adv, IDESC, 1);
+                    } else if (CONCAT) {
+                        umma_tf32(acc, a_hi + adv, w_hi + adv, IDESC_CAT, keep);   // [A hi W hi^T | A hi W lo^T]
+                        umma_tf32(acc + BN, a_lo + adv, w_hi + adv, IDESC, 1);      // the other small term
                     } else {
                         umma_tf32(acc, a_hi + adv, w_lo + adv, IDESC, keep);
                         umma_tf32(acc, a_lo + adv, w_hi + adv, IDESC, 1);
@@ -386,9 +396,14 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                 }
                 // frees the stage (in both CTAs of a pair) once these products have read it
                 if (PAIR) umma_commit_pair(empty_bar(s)); else umma_commit(empty_bar(s));
-                if (kb - chunk * args.chunk_kb == args.chunk_kb - 1 || kb == num_kb - 1) {
+                if (in_chunk == kChunkKb - 1 || kb == num_kb - 1) {
                     if (PAIR) umma_commit_pair(acc_full_bar(buf)); else umma_commit(acc_full_bar(buf));
+                    in_chunk = 0;
+                    ++chunk;
+                } else {
+                    ++in_chunk;
                 }
+                if (++s == STAGES) { s = 0; full_parity ^= 1u; }
             }
         }
     } else {
@@ -400,7 +415,7 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
 #pragma unroll
         for (int j = 0; j < ACC_REGS; ++j) acc[j] = 0.f;
         bool ok = true;
-        const int n_chunks = (num_kb + args.chunk_kb - 1) / args.chunk_kb;
+        const int n_chunks = (num_kb + kChunkKb - 1) / kChunkKb;
 #pragma unroll 1
         for (int chunk = 0; chunk < n_chunks; ++chunk) {
             const int buf = chunk & 1;
@@ -419,6 +434,11 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
 #pragma unroll
             for (int c = 0; c < ACC_REGS; c += 32) {
                 float v[32];
+                if (CONCAT) {            // the small terms first
+                    tmem_ld32(src + BN + c, v);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) acc[c + j] += v[j];
+                }
                 tmem_ld32(src + c, v);   // all lanes take part (sync.aligned)
 #pragma unroll
                 for (int j = 0; j < 32; ++j) acc[c + j] += v[j];
@@ -796,8 +816,6 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     if (const char* e = std::getenv("SAMA_TC_GROUP")) { const int g = std::atoi(e); if (g >= 1 && g <= a.tiles_n) a.group_n = g; }
     dim3 grid(a.tiles_m * a.tiles_n * (pair ? 2 : 1), 1, nbr * a.splits);
     KernelScope scope(ctx, SAMA_K_GEMM_TF32X3, L.layer, st);
-    a.chunk_kb = kChunkKb;
-    if (const char* e = std::getenv("SAMA_TC_CHUNK")) { const int c = std::atoi(e); if (c >= 1) a.chunk_kb = c; }
     // eight epilogue warps (two per lane quarter, each taking half of the columns) except on the 16-wide tile
     if (pair) {
         if (bn == 64) return launch_tc<64, true, 8>(maps, a, grid, st);
