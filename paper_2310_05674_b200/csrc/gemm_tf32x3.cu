@@ -222,13 +222,14 @@ struct TcArgs {
     const float* mask;     // [M][ldm] or null: results are zeroed where mask <= 0
     int ldm;
     int tiles_m, tiles_n, group_n;
-    int splits, kb_per_split;  // split-K: grid.z = 2 * splits, each CTA takes kb_per_split k-blocks
-    float* ws;                 // split-K partial tiles [2 * tiles][splits][BM][BN]
-    int* counters;             // split-K arrival counters [2 * tiles], zero between launches
+    int branches;          // 1 or 2; a work item is (branch, tile)
     uint32_t tx_bytes;     // bytes the four copies of one k-block deliver
     int32_t* status;
 };
 
+// Persistent kernel: CTA (or CTA pair) u of U works on tiles u, u + U, u + 2U, ... of the layer; the copy
+// pipeline and the two accumulators keep running across tiles, so the stores of one tile overlap the
+// products of the next.
 // PAIR = true: two CTAs of a cluster work on one 256 x BN tile.  Each stages its own 128 rows of A and half of
 // the W tile; the leader CTA issues cta_group::2 products that read both CTAs' shared memory and write both
 // CTAs' tensor memory.  Per CTA and flop that is fewer operand bytes than two independent 128 x BN tiles.
@@ -256,7 +257,7 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // tiles need 1024-byte alignment
-    const uint32_t bars = base + STAGES * STAGE;                   // full[STAGES], empty[STAGES], accum, tmem slot
+    const uint32_t bars = base + STAGES * STAGE;                   // full[STAGES], empty[STAGES], accumulators, tmem slot
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
     auto acc_full_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };        // chunk in accumulator b is complete
@@ -268,30 +269,28 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     volatile uint32_t* tmem_ptr_slot =
         reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
 
-    const uint32_t last_slot = abort_slot + 4;
-    volatile uint32_t* last_flag =
-        reinterpret_cast<volatile uint32_t*>(smem_raw + (last_slot - smem_u32(smem_raw)));
-
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int br = blockIdx.z / args.splits, split = blockIdx.z - br * args.splits;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;  // 0 = leader of the pair
-    const int tile_id = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
-    // Tile order: CTAs that run together cover all M-tiles of a group of `group_n` N-tiles, so one wave
-    // re-uses a bounded set of W tiles and every A tile from L2 instead of sweeping all of W.
-    int tile_m, tile_n;
-    {
+    const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int n_units = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const int tiles_per_branch = args.tiles_m * args.tiles_n;
+    const int n_items = tiles_per_branch * args.branches;
+    const int num_kb = args.num_kb;
+    // Work item -> branch and tile origin.  Tile order inside a branch: items that run together cover all
+    // M-tiles of a group of `group_n` N-tiles, so one wave re-uses a bounded set of W tiles and every A tile
+    // from L2 instead of sweeping all of W.
+    auto locate = [&](int item, int& br, int& m0, int& n0) {
+        br = item / tiles_per_branch;
+        const int tile_id = item - br * tiles_per_branch;
         const int per_group = args.group_n * args.tiles_m;
         const int group = tile_id / per_group, rem = tile_id - group * per_group;
         const int first_n = group * args.group_n;
         const int gsz = min(args.group_n, args.tiles_n - first_n);
-        tile_n = first_n + rem % gsz;
-        tile_m = rem / gsz;
-    }
-    const int m0 = tile_m * (PAIR ? 2 * BM : BM) + (int)rank * BM, n0 = tile_n * BN;
-    const int nw0 = n0 + (int)rank * WROWS;  // first W row this CTA stages
-    // this CTA's share of the contraction (the host guarantees at least one k-block per split)
-    const int kb_begin = split * args.kb_per_split;
-    const int num_kb = min(args.kb_per_split, args.num_kb - kb_begin);
+        const int tile_n = first_n + rem % gsz;
+        const int tile_m = rem / gsz;
+        m0 = tile_m * (PAIR ? 2 * BM : BM) + (int)rank * BM;
+        n0 = tile_n * BN;
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -326,84 +325,93 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     if (warp == 0) {
         // ---------------------------------------------------------- TMA producer
         if (lane == 0) {
-            int issued = 0;
-            const int za = args.shared_a ? 0 : br;
+            int issued = 0;  // k-blocks copied so far, over all of this CTA's tiles
             int s = 0;
             uint32_t empty_parity = 1;  // parity of the phase that frees stage s for its next round
-            for (int kb = 0; kb < num_kb; ++kb) {
-                if (kb >= STAGES && !mbar_wait(empty_bar(s), empty_parity, abort_flag)) { raise_timeout(); break; }
-                const uint32_t st = base + s * STAGE;
-                const int kx = (kb_begin + kb) * BKF;
-                if (PAIR) {
-                    // both CTAs' copies complete on the leader's barrier, which the leader arms for all of them
-                    const uint32_t lbar = full_bar(s) & kPeerBitMask;
-                    if (rank == 0) mbar_expect_tx(full_bar(s), args.tx_bytes);
-                    tma_load_3d_pair(st, &map_a_hi, lbar, kx, m0, za);
-                    tma_load_3d_pair(st + A_BYTES, &map_a_lo, lbar, kx, m0, za);
-                    tma_load_3d_pair(st + 2 * A_BYTES, &map_w_hi, lbar, kx, nw0, br);
-                    tma_load_3d_pair(st + 2 * A_BYTES + W_BYTES, &map_w_lo, lbar, kx, nw0, br);
-                } else {
-                    mbar_expect_tx(full_bar(s), args.tx_bytes);
-                    tma_load_3d(st, &map_a_hi, full_bar(s), kx, m0, za);
-                    tma_load_3d(st + A_BYTES, &map_a_lo, full_bar(s), kx, m0, za);
-                    tma_load_3d(st + 2 * A_BYTES, &map_w_hi, full_bar(s), kx, n0, br);
-                    tma_load_3d(st + 2 * A_BYTES + W_BYTES, &map_w_lo, full_bar(s), kx, n0, br);
+            bool ok = true;
+            for (int item = unit; item < n_items && ok; item += n_units) {
+                int br, m0, n0;
+                locate(item, br, m0, n0);
+                const int nw0 = n0 + (int)rank * WROWS;  // first W row this CTA stages
+                const int za = args.shared_a ? 0 : br;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (issued >= STAGES && !mbar_wait(empty_bar(s), empty_parity, abort_flag)) { raise_timeout(); ok = false; break; }
+                    const uint32_t st = base + s * STAGE;
+                    const int kx = kb * BKF;
+                    if (PAIR) {
+                        // both CTAs' copies complete on the leader's barrier, which the leader arms for all of them
+                        const uint32_t lbar = full_bar(s) & kPeerBitMask;
+                        if (rank == 0) mbar_expect_tx(full_bar(s), args.tx_bytes);
+                        tma_load_3d_pair(st, &map_a_hi, lbar, kx, m0, za);
+                        tma_load_3d_pair(st + A_BYTES, &map_a_lo, lbar, kx, m0, za);
+                        tma_load_3d_pair(st + 2 * A_BYTES, &map_w_hi, lbar, kx, nw0, br);
+                        tma_load_3d_pair(st + 2 * A_BYTES + W_BYTES, &map_w_lo, lbar, kx, nw0, br);
+                    } else {
+                        mbar_expect_tx(full_bar(s), args.tx_bytes);
+                        tma_load_3d(st, &map_a_hi, full_bar(s), kx, m0, za);
+                        tma_load_3d(st + A_BYTES, &map_a_lo, full_bar(s), kx, m0, za);
+                        tma_load_3d(st + 2 * A_BYTES, &map_w_hi, full_bar(s), kx, n0, br);
+                        tma_load_3d(st + 2 * A_BYTES + W_BYTES, &map_w_lo, full_bar(s), kx, n0, br);
+                    }
+                    ++issued;
+                    if (++s == STAGES) { s = 0; empty_parity ^= 1u; }
                 }
-                issued = kb + 1;
-                if (++s == STAGES) { s = 0; empty_parity ^= 1u; }
             }
             if (*abort_flag && rank == 0) {
                 // let the copies already issued land before the CTA's shared memory goes away
-                for (int kb = (issued > STAGES ? issued - STAGES : 0); kb < issued; ++kb)
-                    mbar_wait(full_bar(kb % STAGES), (kb / STAGES) & 1);
+                for (int i = (issued > STAGES ? issued - STAGES : 0); i < issued; ++i)
+                    mbar_wait(full_bar(i % STAGES), (i / STAGES) & 1);
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (the leader's, for a pair)
         if (lane == 0 && rank == 0) {
             bool ok = true;
-            int s = 0, in_chunk = 0, chunk = 0;
+            int s = 0, chunk = 0;  // chunk counts over all of this CTA's tiles: accumulator = chunk & 1
             uint32_t full_parity = 0;
-            for (int kb = 0; kb < num_kb && ok; ++kb) {
-                const int buf = chunk & 1;
-                const bool chunk_first = in_chunk == 0;
-                if (chunk_first && chunk >= 2) {
-                    // the epilogue warps have drained this accumulator's previous chunk
-                    if (!mbar_wait(acc_empty_bar(buf), ((chunk >> 1) - 1) & 1, abort_flag)) { raise_timeout(); ok = false; break; }
-                }
-                if (!mbar_wait(full_bar(s), full_parity, abort_flag)) { raise_timeout(); ok = false; break; }
-                tc_fence_after();
-                const uint32_t st = base + s * STAGE;
-                const uint32_t acc = tmem_base + (uint32_t)buf * ACC_COLS;
-                const uint64_t a_hi = make_desc(st), a_lo = make_desc(st + A_BYTES);
-                const uint64_t w_hi = make_desc(st + 2 * A_BYTES), w_lo = make_desc(st + 2 * A_BYTES + W_BYTES);
-#pragma unroll
-                for (int k = 0; k < BKF / UMMA_K; ++k) {
-                    const uint64_t adv = (uint64_t)((k * UMMA_K * 4) >> 4);  // 32 bytes per k-step inside the swizzled row
-                    const uint32_t keep = (chunk_first && k == 0) ? 0u : 1u;  // a chunk starts from zero
-                    if (PAIR) {
-                        umma_tf32_pair(acc, a_hi + adv, w_lo + adv, IDESC, keep);
-                        umma_tf32_pair(acc, a_lo + adv, w_hi + adv, IDESC, 1);
-                        umma_tf32_pair(acc, a_hi + adv, w_hi + adv, IDESC, 1);
-                    } else if (CONCAT) {
-                        umma_tf32(acc, a_hi + adv, w_hi + adv, IDESC_CAT, keep);   // [A hi W hi^T | A hi W lo^T]
-                        umma_tf32(acc + BN, a_lo + adv, w_hi + adv, IDESC, 1);      // the other small term
-                    } else {
-                        umma_tf32(acc, a_hi + adv, w_lo + adv, IDESC, keep);
-                        umma_tf32(acc, a_lo + adv, w_hi + adv, IDESC, 1);
-                        umma_tf32(acc, a_hi + adv, w_hi + adv, IDESC, 1);
+            for (int item = unit; item < n_items && ok; item += n_units) {
+                int in_chunk = 0;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    const int buf = chunk & 1;
+                    const bool chunk_first = in_chunk == 0;
+                    if (chunk_first && chunk >= 2) {
+                        // the epilogue warps have drained this accumulator's previous chunk
+                        if (!mbar_wait(acc_empty_bar(buf), ((chunk >> 1) - 1) & 1, abort_flag)) { raise_timeout(); ok = false; break; }
                     }
+                    if (!mbar_wait(full_bar(s), full_parity, abort_flag)) { raise_timeout(); ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t st = base + s * STAGE;
+                    const uint32_t acc = tmem_base + (uint32_t)buf * ACC_COLS;
+                    const uint64_t a_hi = make_desc(st), a_lo = make_desc(st + A_BYTES);
+                    const uint64_t w_hi = make_desc(st + 2 * A_BYTES), w_lo = make_desc(st + 2 * A_BYTES + W_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BKF / UMMA_K; ++k) {
+                        const uint64_t adv = (uint64_t)((k * UMMA_K * 4) >> 4);  // 32 bytes per k-step inside the swizzled row
+                        const uint32_t keep = (chunk_first && k == 0) ? 0u : 1u;  // a chunk starts from zero
+                        if (PAIR) {
+                            umma_tf32_pair(acc, a_hi + adv, w_lo + adv, IDESC, keep);
+                            umma_tf32_pair(acc, a_lo + adv, w_hi + adv, IDESC, 1);
+                            umma_tf32_pair(acc, a_hi + adv, w_hi + adv, IDESC, 1);
+                        } else if (CONCAT) {
+                            umma_tf32(acc, a_hi + adv, w_hi + adv, IDESC_CAT, keep);   // [A hi W hi^T | A hi W lo^T]
+                            umma_tf32(acc + BN, a_lo + adv, w_hi + adv, IDESC, 1);      // the other small term
+                        } else {
+                            umma_tf32(acc, a_hi + adv, w_lo + adv, IDESC, keep);
+                            umma_tf32(acc, a_lo + adv, w_hi + adv, IDESC, 1);
+                            umma_tf32(acc, a_hi + adv, w_hi + adv, IDESC, 1);
+                        }
+                    }
+                    // frees the stage (in both CTAs of a pair) once these products have read it
+                    if (PAIR) umma_commit_pair(empty_bar(s)); else umma_commit(empty_bar(s));
+                    if (in_chunk == kChunkKb - 1 || kb == num_kb - 1) {
+                        if (PAIR) umma_commit_pair(acc_full_bar(buf)); else umma_commit(acc_full_bar(buf));
+                        in_chunk = 0;
+                        ++chunk;
+                    } else {
+                        ++in_chunk;
+                    }
+                    if (++s == STAGES) { s = 0; full_parity ^= 1u; }
                 }
-                // frees the stage (in both CTAs of a pair) once these products have read it
-                if (PAIR) umma_commit_pair(empty_bar(s)); else umma_commit(empty_bar(s));
-                if (in_chunk == kChunkKb - 1 || kb == num_kb - 1) {
-                    if (PAIR) umma_commit_pair(acc_full_bar(buf)); else umma_commit(acc_full_bar(buf));
-                    in_chunk = 0;
-                    ++chunk;
-                } else {
-                    ++in_chunk;
-                }
-                if (++s == STAGES) { s = 0; full_parity ^= 1u; }
             }
         }
     } else {
@@ -411,146 +419,102 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         const int q = warp & 3;            // a warp may only touch TMEM lanes [32 q, 32 q + 32)
         const int col0 = ((warp - 2) >> 2) * CPW;  // with eight epilogue warps, two share a lane quarter and split the columns
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)col0;
-        float acc[ACC_REGS];
-#pragma unroll
-        for (int j = 0; j < ACC_REGS; ++j) acc[j] = 0.f;
-        bool ok = true;
         const int n_chunks = (num_kb + kChunkKb - 1) / kChunkKb;
+        int chunk = 0;  // counts over all of this CTA's tiles, like the issuer's
+        bool ok = true;
+        for (int item = unit; item < n_items && ok; item += n_units) {
+            int br, m0, n0;
+            locate(item, br, m0, n0);
+            float acc[ACC_REGS];
+#pragma unroll
+            for (int j = 0; j < ACC_REGS; ++j) acc[j] = 0.f;
 #pragma unroll 1
-        for (int chunk = 0; chunk < n_chunks; ++chunk) {
-            const int buf = chunk & 1;
-            if (lane == 0) {
-                // the chunk is complete when its barrier flips, or never if a producer gave up
-                const long long t0 = clock64();
-                while (!mbar_try(acc_full_bar(buf), (chunk >> 1) & 1)) {
-                    if (*abort_flag) { ok = false; break; }
-                    if (clock64() - t0 > 2 * kWaitCycles) { raise_timeout(); ok = false; break; }
+            for (int c = 0; c < n_chunks; ++c, ++chunk) {
+                const int buf = chunk & 1;
+                if (lane == 0) {
+                    // the chunk is complete when its barrier flips, or never if a producer gave up
+                    const long long t0 = clock64();
+                    while (!mbar_try(acc_full_bar(buf), (chunk >> 1) & 1)) {
+                        if (*abort_flag) { ok = false; break; }
+                        if (clock64() - t0 > 2 * kWaitCycles) { raise_timeout(); ok = false; break; }
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t src = lane_addr + (uint32_t)buf * ACC_COLS;
+#pragma unroll
+                for (int cc = 0; cc < ACC_REGS; cc += 32) {
+                    float v[32];
+                    if (CONCAT) {            // the small terms first
+                        tmem_ld32(src + BN + cc, v);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) acc[cc + j] += v[j];
+                    }
+                    tmem_ld32(src + cc, v);   // all lanes take part (sync.aligned)
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) acc[cc + j] += v[j];
+                }
+                // this warp's reads are done: hand the accumulator back to the MMA issuer
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (PAIR) mbar_arrive_cluster(acc_empty_bar(buf) & kPeerBitMask); else mbar_arrive(acc_empty_bar(buf));
                 }
             }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
-            tc_fence_after();
-            const uint32_t src = lane_addr + (uint32_t)buf * ACC_COLS;
-#pragma unroll
-            for (int c = 0; c < ACC_REGS; c += 32) {
-                float v[32];
-                if (CONCAT) {            // the small terms first
-                    tmem_ld32(src + BN + c, v);
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) acc[c + j] += v[j];
-                }
-                tmem_ld32(src + c, v);   // all lanes take part (sync.aligned)
-#pragma unroll
-                for (int j = 0; j < 32; ++j) acc[c + j] += v[j];
-            }
-            // this warp's reads are done: hand the accumulator back to the MMA issuer
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0 && chunk + 2 < n_chunks) {
-                if (PAIR) mbar_arrive_cluster(acc_empty_bar(buf) & kPeerBitMask); else mbar_arrive(acc_empty_bar(buf));
-            }
-        }
-        // the epilogue warps proceed together or not at all (they meet again at named barrier 1)
-        volatile uint32_t* ok_slots = last_flag + 1;
-        if (lane == 0) ok_slots[warp - 2] = ok ? 1u : 0u;
-        asm volatile("bar.sync 1, %0;" ::"n"(32 * EPI) : "memory");
-        {
-            uint32_t all = 1u;
-#pragma unroll
-            for (int w = 0; w < EPI; ++w) all &= ok_slots[w];
-            ok = all != 0;
-        }
-        if (ok) {
+            // the tile's sum is in registers; the products of the next tile already run while it is stored
             const int row = q * 32 + lane;
             const int m = m0 + row;
             const float* bias = br ? args.bias[1] : args.bias[0];
-            // Split-K: every CTA of a tile stores its raw partial; the last one to arrive adds the
-            // partials in split order (so the sum does not depend on which CTA that is) and finishes.
-            const float* part = nullptr;
-            bool finish = true;
-            if (args.splits > 1) {
-                const int tile_lin = br * (args.tiles_m * args.tiles_n) + (int)blockIdx.x;
-                float* base_ws = args.ws + (int64_t)tile_lin * args.splits * (BM * BN);
-                float* mine = base_ws + ((int64_t)split * BM + row) * BN + col0;
-#pragma unroll
-                for (int c = 0; c < CPW; c += 4)
-                    __stcg(reinterpret_cast<float4*>(mine + c), make_float4(acc[c], acc[c + 1], acc[c + 2], acc[c + 3]));
-                __threadfence();
-                asm volatile("bar.sync 1, %0;" ::"n"(32 * EPI) : "memory");
-                if (warp == 2 && lane == 0) {
-                    const int prev = atomicAdd(args.counters + tile_lin, 1);
-                    const bool is_last = (prev == args.splits - 1);
-                    if (is_last) args.counters[tile_lin] = 0;  // every CTA of the tile has arrived
-                    *last_flag = is_last ? 1u : 0u;
-                }
-                asm volatile("bar.sync 1, %0;" ::"n"(32 * EPI) : "memory");
-                finish = (*last_flag != 0);
-                if (finish) __threadfence();
-                part = base_ws + (int64_t)row * BN + col0;
-            }
-            if (finish) {
+            if (m < args.M) {
 #pragma unroll
                 for (int c = 0; c < CPW; c += 16) {
                     float v[16];
-                    if (part) {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) v[j] = 0.f;
-                        for (int sp = 0; sp < args.splits; ++sp) {
-                            const float4* src = reinterpret_cast<const float4*>(part + (int64_t)sp * (BM * BN) + c);
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const float4 t = __ldcg(src + j);
-                                v[4 * j] += t.x; v[4 * j + 1] += t.y; v[4 * j + 2] += t.z; v[4 * j + 3] += t.w;
-                            }
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) v[j] = acc[c + j];
-                    }
+                    for (int j = 0; j < 16; ++j) v[j] = acc[c + j];
                     const int n = n0 + col0 + c;
-                    if (m < args.M) {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            float x = v[j] + ((bias != nullptr && n + j < args.N) ? bias[n + j] : 0.f);
-                            if (args.relu && x < 0.f) x = 0.f;
-                            v[j] = x;
-                        }
-                        if (args.mask) {  // backward pass: the derivative passes only where the forward activation was positive
-                            const float* mk = args.mask + (int64_t)m * args.ldm + n;
+                    for (int j = 0; j < 16; ++j) {
+                        float x = v[j] + ((bias != nullptr && n + j < args.N) ? bias[n + j] : 0.f);
+                        if (args.relu && x < 0.f) x = 0.f;
+                        v[j] = x;
+                    }
+                    if (args.mask) {  // backward pass: the derivative passes only where the forward activation was positive
+                        const float* mk = args.mask + (int64_t)m * args.ldm + n;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (n + j < args.N && !(mk[j] > 0.f)) v[j] = 0.f;
+                    }
+                    if (args.last || args.both) {
+                        float* dst = (br ? args.out_f32[1] : args.out_f32[0]) + (int64_t)m * args.ldc + n;
+                        if (n + 15 < args.N && (args.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                reinterpret_cast<float4*>(dst)[j] =
+                                    make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                        } else {
 #pragma unroll
                             for (int j = 0; j < 16; ++j)
-                                if (n + j < args.N && !(mk[j] > 0.f)) v[j] = 0.f;
+                                if (n + j < args.N) dst[j] = v[j];
                         }
-                        if (args.last || args.both) {
-                            float* dst = (br ? args.out_f32[1] : args.out_f32[0]) + (int64_t)m * args.ldc + n;
-                            if (n + 15 < args.N && (args.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+                    }
+                    if (!args.last && n < args.ld_next) {
+                        // columns in [N, ld_next) are the next layer's zero padding along K
+                        const int64_t off = ((int64_t)br * args.M + m) * args.ld_next + n;
+                        float hi[16], lo[16];
 #pragma unroll
-                                for (int j = 0; j < 4; ++j)
-                                    reinterpret_cast<float4*>(dst)[j] =
-                                        make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 16; ++j)
-                                    if (n + j < args.N) dst[j] = v[j];
-                            }
+                        for (int j = 0; j < 16; ++j) {
+                            const float x = (n + j < args.N) ? v[j] : 0.f;
+                            hi[j] = to_tf32(x);
+                            lo[j] = to_tf32(x - hi[j]);
                         }
-                        if (!args.last && n < args.ld_next) {
-                            // columns in [N, ld_next) are the next layer's zero padding along K
-                            const int64_t off = ((int64_t)br * args.M + m) * args.ld_next + n;
-                            float hi[16], lo[16];
+                        float4* dh = reinterpret_cast<float4*>(args.out_hi + off);
+                        float4* dl = reinterpret_cast<float4*>(args.out_lo + off);
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) {
-                                const float x = (n + j < args.N) ? v[j] : 0.f;
-                                hi[j] = to_tf32(x);
-                                lo[j] = to_tf32(x - hi[j]);
-                            }
-                            float4* dh = reinterpret_cast<float4*>(args.out_hi + off);
-                            float4* dl = reinterpret_cast<float4*>(args.out_lo + off);
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                dh[j] = make_float4(hi[4 * j], hi[4 * j + 1], hi[4 * j + 2], hi[4 * j + 3]);
-                                dl[j] = make_float4(lo[4 * j], lo[4 * j + 1], lo[4 * j + 2], lo[4 * j + 3]);
-                            }
+                        for (int j = 0; j < 4; ++j) {
+                            dh[j] = make_float4(hi[4 * j], hi[4 * j + 1], hi[4 * j + 2], hi[4 * j + 3]);
+                            dl[j] = make_float4(lo[4 * j], lo[4 * j + 1], lo[4 * j + 2], lo[4 * j + 3]);
                         }
                     }
                 }
@@ -679,18 +643,39 @@ bool make_map(CUtensorMap* map, const float* base, int ld, int64_t rows, int sla
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Launches the persistent kernel on min(work items, co-resident CTAs or CTA pairs) units.
 template <int BN, bool PAIR, int EPI>
-cudaError_t launch_tc(const CUtensorMap maps[4], const TcArgs& a, dim3 grid, cudaStream_t st) {
+cudaError_t launch_tc(const CUtensorMap maps[4], const TcArgs& a, int items, int sm_count, cudaStream_t st) {
     constexpr int kSmem = smem_bytes(PAIR ? BN / 2 : BN);
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tf32x3_kernel<BN, PAIR, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kSmem);
+    static int max_units = 0;  // one CTA per SM (shared memory); pairs: what the cluster scheduler can co-schedule
+    if (max_units == 0) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_tf32x3_kernel<BN, PAIR, EPI>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
         if (e != cudaSuccess) return e;
-        configured = true;
+        int units = sm_count;
+        if (PAIR) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(2 * (sm_count / 2));
+            cfg.blockDim = dim3(threads_for(EPI));
+            cfg.dynamicSmemBytes = kSmem;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 2;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            int clusters = 0;
+            e = cudaOccupancyMaxActiveClusters(&clusters, gemm_tf32x3_kernel<BN, PAIR, EPI>, &cfg);
+            if (e != cudaSuccess) return e;
+            units = clusters < sm_count / 2 ? clusters : sm_count / 2;
+        }
+        if (units < 1) return cudaErrorLaunchOutOfResources;
+        max_units = units;
     }
-    return launch_clustered(PAIR ? 2 : 1, gemm_tf32x3_kernel<BN, PAIR, EPI>, grid, dim3(threads_for(EPI)), (size_t)kSmem, st,
-                            maps[0], maps[1], maps[2], maps[3], a);
+    const int units = items < max_units ? items : max_units;
+    return launch_clustered(PAIR ? 2 : 1, gemm_tf32x3_kernel<BN, PAIR, EPI>, dim3(units * (PAIR ? 2 : 1)),
+                            dim3(threads_for(EPI)), (size_t)kSmem, st, maps[0], maps[1], maps[2], maps[3], a);
 }
 
 inline int round_up32(int x) { return (x + 31) & ~31; }
@@ -738,30 +723,13 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     // (Hidden layers never take 16: their tiles must also write the zero padding up to round_up32(N).)
     const int nbr = L.branches == 1 ? 1 : 2;  // the direct gradient runs a single branch
     const int64_t tiles128 = (int64_t)((L.M + BM - 1) / BM) * ((L.N + 127) / 128) * nbr;
-    // Split-K (several CTAs per tile, partials added in split order by the last CTA to arrive) exists for
-    // contractions that are long relative to the grid, but measured slower than 64-wide tiles on every
-    // workload here (the partial-tile round trip costs more than the idle SMs), so it is off unless the
-    // SAMA_TC_SPLITS environment variable asks for it.
     const bool narrow_last = L.last && L.N <= 16;
     int bn = narrow_last ? 16 : ((L.N <= 64 || tiles128 < ctx->sm_count) ? 64 : 128);
     if (ctx->tile_override == 64 || ctx->tile_override == 128) bn = ctx->tile_override;
-    const int num_kb_total = Kp / BKF;
-    int splits = 1;
-    {
-        const int64_t tiles = (int64_t)((L.M + BM - 1) / BM) * ((L.N + bn - 1) / bn) * nbr;
-        int want = 1;
-        if (const char* e = std::getenv("SAMA_TC_SPLITS")) want = std::atoi(e);
-        if (want > 8) want = 8;
-        const int by_k = num_kb_total / 4;  // at least 4 k-blocks per split
-        if (want > by_k) want = by_k;
-        while (want > 1 && (size_t)tiles * want * BM * bn > ctx->tc_ws_floats) --want;
-        if (tiles > kTcCounters) want = 1;
-        if (want > 1 && ctx->tc_ws && ctx->tc_counters) splits = want;
-    }
     // CTA pairs (256 x bn tiles): per CTA and flop they stage fewer operand bytes, which is what bounds this
     // kernel -- but only worth it when the pairs still fill the machine (measured: wide4096 and head1024 gain
     // 10 %, mlp3072 loses 4 %).  The widest pair tile whose grid covers every SM is taken.
-    bool pair = !narrow_last && splits == 1 && L.M > BM && L.N >= 128;
+    bool pair = !narrow_last && L.M > BM && L.N >= 128;
     if (const char* e = std::getenv("SAMA_TC_PAIR")) pair = pair && std::atoi(e) != 0;
     if (pair) {
         auto ctas = [&](int w) { return 2 * (int64_t)((L.M + 2 * BM - 1) / (2 * BM)) * ((L.N + w - 1) / w) * nbr; };
@@ -805,26 +773,24 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     a.status = &ctx->scalars->status;
     a.tiles_m = pair ? (L.M + 2 * BM - 1) / (2 * BM) : (L.M + BM - 1) / BM;
     a.tiles_n = (L.N + bn - 1) / bn;
+    a.branches = nbr;
     // about one wave of CTAs per group: group_n N-tiles x all M-tiles
-    a.kb_per_split = (num_kb_total + splits - 1) / splits;
-    a.splits = (num_kb_total + a.kb_per_split - 1) / a.kb_per_split;  // no empty split
-    a.ws = ctx->tc_ws;
-    a.counters = ctx->tc_counters;
     a.group_n = ctx->sm_count / a.tiles_m;
     if (a.group_n < 1) a.group_n = 1;
     if (a.group_n > a.tiles_n) a.group_n = a.tiles_n;
     if (const char* e = std::getenv("SAMA_TC_GROUP")) { const int g = std::atoi(e); if (g >= 1 && g <= a.tiles_n) a.group_n = g; }
-    dim3 grid(a.tiles_m * a.tiles_n * (pair ? 2 : 1), 1, nbr * a.splits);
+    const int items = a.tiles_m * a.tiles_n * nbr;
+    const int sms = ctx->sm_count;
     KernelScope scope(ctx, SAMA_K_GEMM_TF32X3, L.layer, st);
     // eight epilogue warps (two per lane quarter, each taking half of the columns) except on the 16-wide tile
     if (pair) {
-        if (bn == 64) return launch_tc<64, true, 8>(maps, a, grid, st);
-        if (bn == 256) return launch_tc<256, true, 8>(maps, a, grid, st);
-        return launch_tc<128, true, 8>(maps, a, grid, st);
+        if (bn == 64) return launch_tc<64, true, 8>(maps, a, items, sms, st);
+        if (bn == 256) return launch_tc<256, true, 8>(maps, a, items, sms, st);
+        return launch_tc<128, true, 8>(maps, a, items, sms, st);
     }
-    if (bn == 16) return launch_tc<16, false, 4>(maps, a, grid, st);
-    if (bn == 64) return launch_tc<64, false, 8>(maps, a, grid, st);
-    return launch_tc<128, false, 8>(maps, a, grid, st);
+    if (bn == 16) return launch_tc<16, false, 4>(maps, a, items, sms, st);
+    if (bn == 64) return launch_tc<64, false, 8>(maps, a, items, sms, st);
+    return launch_tc<128, false, 8>(maps, a, items, sms, st);
 }
 
 }  // namespace sama

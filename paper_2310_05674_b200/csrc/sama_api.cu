@@ -394,10 +394,6 @@ int sama_create(sama_ctx** out, int device, int64_t max_n, int32_t max_batch, co
         ok = ok && cudaMalloc(&ctx->mg_ws, sizeof(float) * ctx->mg_ws_floats) == cudaSuccess;
         ctx->mg_tc_floats = meta_grad_tc_floats(mlp, max_batch);
         ok = ok && cudaMalloc(&ctx->mg_tc, sizeof(float) * ctx->mg_tc_floats) == cudaSuccess;
-        ctx->tc_ws_floats = (size_t)8 << 20;  // 32 MiB of split-K partial tiles
-        ok = ok && cudaMalloc(&ctx->tc_ws, sizeof(float) * ctx->tc_ws_floats) == cudaSuccess &&
-             cudaMalloc(&ctx->tc_counters, sizeof(int) * kTcCounters) == cudaSuccess &&
-             cudaMemset(ctx->tc_counters, 0, sizeof(int) * kTcCounters) == cudaSuccess;
         if (ok && amax > 0)
             ok = cudaMalloc(&ctx->a_split[0], sizeof(float) * 2 * ctx->a_split_half) == cudaSuccess &&
                  cudaMalloc(&ctx->a_split[1], sizeof(float) * 2 * ctx->a_split_half) == cudaSuccess;
@@ -423,10 +419,8 @@ int sama_destroy(sama_ctx* ctx) {
     cudaFree(ctx->w_split);
     cudaFree(ctx->a_split[0]);
     cudaFree(ctx->a_split[1]);
-    cudaFree(ctx->tc_ws);
     cudaFree(ctx->mg_ws);
     cudaFree(ctx->mg_tc);
-    cudaFree(ctx->tc_counters);
     cudaFree(ctx->stage);
     if (ctx->prof) {
         for (auto& r : ctx->prof->records) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }

@@ -10,8 +10,7 @@
 namespace sama {
 
 constexpr int kMaxLayers = 16;
-constexpr int kMaxPartials = 4096;
-constexpr int kTcCounters = 4096;   // split-K arrival counters (tiles of one layer, both branches)  // upper bound on the grid of the reduction kernels
+constexpr int kMaxPartials = 4096;  // upper bound on the grid of the reduction kernels
 
 // Device scalars owned by a context.
 struct DeviceScalars {
@@ -86,9 +85,6 @@ struct sama_ctx {
     float* w_split;                // device [hi, lo][2 branches][slab]: every layer's W, rows padded to 32
     float* a_split[2];             // device, ping-pong: [2][2][max_batch][round32(max hidden)]
     size_t x_split_half, w_split_half, a_split_half;  // floats per hi (or lo) part; 0 = path unavailable
-    float* tc_ws;                  // device: split-K partial tiles of the tensor-core path
-    size_t tc_ws_floats;
-    int* tc_counters;              // device [kTcCounters], zero between launches
     float* mg_ws;                  // device: workspace of the direct gradient (activations, dz, losses)
     size_t mg_ws_floats;
     float* mg_tc;                  // device: TF32 operand buffers of the direct gradient's tensor-core path

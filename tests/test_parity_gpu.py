@@ -286,11 +286,14 @@ def test_step_is_bitwise_reproducible(gemm_mode):
             assert r["sumsq"] == runs[0]["sumsq"] and r["eps_fd"] == runs[0]["eps_fd"]
 
 
-def test_split_k_option_matches_and_is_reproducible(monkeypatch):
-    """The optional split of the contraction over several CTAs per tile (SAMA_TC_SPLITS) adds its
-    partial tiles in a fixed order: same parity bar, bitwise repeatable."""
-    monkeypatch.setenv("SAMA_TC_SPLITS", "3")
-    cfg, w = W.custom_mlp((2048, 512, 300, 40), 200, seed=8)
+@pytest.mark.parametrize("pairs", ["1", "0"])
+def test_several_tiles_per_cta(monkeypatch, pairs):
+    """More output tiles than SMs: every CTA (or CTA pair; SAMA_TC_PAIR=0 forces single CTAs) of the
+    persistent tensor-core kernel walks several tiles, with its copy pipeline and accumulators running
+    across the tile boundary; the contraction (10 k-blocks) ends on a short chunk.  Same parity bar,
+    bitwise repeatable."""
+    monkeypatch.setenv("SAMA_TC_PAIR", pairs)
+    cfg, w = W.custom_mlp((300, 2304, 40), 1200, seed=8)
     check_step(cfg, w, B.Adam(), 1.0, gemm_mode=2)
     with Ctx(cfg.n_params, cfg.batch, cfg.dims, 2) as ctx:
         a = run_step(ctx, cfg, w, B.Adam(), 1.0)
