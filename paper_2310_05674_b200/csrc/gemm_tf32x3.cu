@@ -57,7 +57,10 @@ __host__ __device__ constexpr int stage_bytes(int wrows) { return 2 * BM * BKF *
 __host__ __device__ constexpr int stages_for(int wrows) {
     return (200 * 1024) / stage_bytes(wrows) > 5 ? 5 : (200 * 1024) / stage_bytes(wrows);
 }
-__host__ __device__ constexpr int smem_bytes(int wrows) { return stages_for(wrows) * stage_bytes(wrows) + 1024 + 256; }
+constexpr int kStoreStageBytes = 32 * 32 * 4;  // per epilogue warp: a 32 x 32 fp32 block on its way to row-contiguous stores
+__host__ __device__ constexpr int smem_bytes(int wrows) {
+    return stages_for(wrows) * stage_bytes(wrows) + 1024 + 256 + 8 * kStoreStageBytes;
+}
 
 // ---------------------------------------------------------------- PTX wrappers
 
@@ -463,58 +466,68 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                 }
             }
             if (!ok) break;
-            // the tile's sum is in registers; the products of the next tile already run while it is stored
-            const int row = q * 32 + lane;
-            const int m = m0 + row;
+            // The tile's sum is in registers; the products of the next tile already run while it is stored.
+            // A thread holds one row; to store whole 128-byte row segments the warp passes each 32 x 32 block
+            // through shared memory (16-byte chunks XOR-swizzled by row: no bank conflicts either way), after
+            // which eight lanes cover one row's 32 columns and an instruction writes four full segments.
+            float4* stg = reinterpret_cast<float4*>(smem_raw + (bars + 256u - smem_u32(smem_raw))) + (warp - 2) * 256;
             const float* bias = br ? args.bias[1] : args.bias[0];
-            if (m < args.M) {
+            float* outf = br ? args.out_f32[1] : args.out_f32[0];
+            const bool vec_f32 = (args.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(outf) & 15u) == 0;
+            const int c4 = lane & 7;
 #pragma unroll
-                for (int c = 0; c < CPW; c += 16) {
-                    float v[16];
+            for (int g = 0; g < ACC_REGS / 32; ++g) {
+                __syncwarp();
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] = acc[c + j];
-                    const int n = n0 + col0 + c;
+                for (int k = 0; k < 8; ++k)
+                    stg[lane * 8 + (k ^ (lane & 7))] =
+                        make_float4(acc[32 * g + 4 * k], acc[32 * g + 4 * k + 1], acc[32 * g + 4 * k + 2], acc[32 * g + 4 * k + 3]);
+                __syncwarp();
+                const int cl = 32 * g + 4 * c4;  // this lane's four columns within the thread's column range
+                const int n = n0 + col0 + cl;
+                if (cl < CPW) {                  // (the 16-wide tile fills only half of the block)
+                    float b[4];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        float x = v[j] + ((bias != nullptr && n + j < args.N) ? bias[n + j] : 0.f);
-                        if (args.relu && x < 0.f) x = 0.f;
-                        v[j] = x;
-                    }
-                    if (args.mask) {  // backward pass: the derivative passes only where the forward activation was positive
-                        const float* mk = args.mask + (int64_t)m * args.ldm + n;
+                    for (int j = 0; j < 4; ++j) b[j] = (bias != nullptr && n + j < args.N) ? bias[n + j] : 0.f;
 #pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (n + j < args.N && !(mk[j] > 0.f)) v[j] = 0.f;
-                    }
-                    if (args.last || args.both) {
-                        float* dst = (br ? args.out_f32[1] : args.out_f32[0]) + (int64_t)m * args.ldc + n;
-                        if (n + 15 < args.N && (args.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+                    for (int i = 0; i < 8; ++i) {
+                        const int rl = 4 * i + (lane >> 3);
+                        const int m = m0 + q * 32 + rl;
+                        const float4 t = stg[rl * 8 + (c4 ^ (rl & 7))];
+                        if (m >= args.M) continue;
+                        float v[4] = {t.x + b[0], t.y + b[1], t.z + b[2], t.w + b[3]};
+                        if (args.relu) {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) v[j] = v[j] < 0.f ? 0.f : v[j];
+                        }
+                        if (args.mask) {  // backward pass: the derivative passes only where the forward activation was positive
+                            const float* mk = args.mask + (int64_t)m * args.ldm + n;
 #pragma unroll
                             for (int j = 0; j < 4; ++j)
-                                reinterpret_cast<float4*>(dst)[j] =
-                                    make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                if (n + j < args.N) dst[j] = v[j];
+                                if (n + j < args.N && !(mk[j] > 0.f)) v[j] = 0.f;
                         }
-                    }
-                    if (!args.last && n < args.ld_next) {
-                        // columns in [N, ld_next) are the next layer's zero padding along K
-                        const int64_t off = ((int64_t)br * args.M + m) * args.ld_next + n;
-                        float hi[16], lo[16];
+                        if (args.last || args.both) {
+                            float* dst = outf + (int64_t)m * args.ldc + n;
+                            if (vec_f32 && n + 3 < args.N) {
+                                *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+                            } else {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const float x = (n + j < args.N) ? v[j] : 0.f;
-                            hi[j] = to_tf32(x);
-                            lo[j] = to_tf32(x - hi[j]);
+                                for (int j = 0; j < 4; ++j)
+                                    if (n + j < args.N) dst[j] = v[j];
+                            }
                         }
-                        float4* dh = reinterpret_cast<float4*>(args.out_hi + off);
-                        float4* dl = reinterpret_cast<float4*>(args.out_lo + off);
+                        if (!args.last && n < args.ld_next) {
+                            // columns in [N, ld_next) are the next layer's zero padding along K
+                            const int64_t off = ((int64_t)br * args.M + m) * args.ld_next + n;
+                            float hi[4], lo[4];
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            dh[j] = make_float4(hi[4 * j], hi[4 * j + 1], hi[4 * j + 2], hi[4 * j + 3]);
-                            dl[j] = make_float4(lo[4 * j], lo[4 * j + 1], lo[4 * j + 2], lo[4 * j + 3]);
+                            for (int j = 0; j < 4; ++j) {
+                                const float x = (n + j < args.N) ? v[j] : 0.f;
+                                hi[j] = to_tf32(x);
+                                lo[j] = to_tf32(x - hi[j]);
+                            }
+                            *reinterpret_cast<float4*>(args.out_hi + off) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                            *reinterpret_cast<float4*>(args.out_lo + off) = make_float4(lo[0], lo[1], lo[2], lo[3]);
                         }
                     }
                 }
@@ -719,25 +732,39 @@ cudaError_t launch_split_transpose_tf32(sama_ctx* ctx, const float* src, int64_t
 // writes fp32 logits.
 cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st) {
     const int Kp = round_up32(L.K);
-    // N-tile: 16 for a narrow last layer; 64 when 128-wide tiles would leave SMs idle; else 128.
-    // (Hidden layers never take 16: their tiles must also write the zero padding up to round_up32(N).)
     const int nbr = L.branches == 1 ? 1 : 2;  // the direct gradient runs a single branch
-    const int64_t tiles128 = (int64_t)((L.M + BM - 1) / BM) * ((L.N + 127) / 128) * nbr;
+    const int num_kb = Kp / BKF;
+    // Tile shape.  A narrow last layer takes the 16-wide tile (hidden layers never do: their tiles must also
+    // write the zero padding up to round_up32(N)).  Otherwise the candidates are single-CTA tiles of 128 x 64
+    // and 128 x 128 and the CTA pair's 256 x 256; the one with the lowest estimate of
+    //   rounds x (k-blocks x time per k-block + time to store a tile),  rounds = ceil(tiles / co-resident units)
+    // is taken.  Times per k-block (microseconds, measured on the three workloads): wider tiles do more
+    // work per staged operand byte, narrower ones fill the machine when the layer has few tiles.
     const bool narrow_last = L.last && L.N <= 16;
-    int bn = narrow_last ? 16 : ((L.N <= 64 || tiles128 < ctx->sm_count) ? 64 : 128);
-    if (ctx->tile_override == 64 || ctx->tile_override == 128) bn = ctx->tile_override;
-    // CTA pairs (256 x bn tiles): per CTA and flop they stage fewer operand bytes, which is what bounds this
-    // kernel -- but only worth it when the pairs still fill the machine (measured: wide4096 and head1024 gain
-    // 10 %, mlp3072 loses 4 %).  The widest pair tile whose grid covers every SM is taken.
-    bool pair = !narrow_last && L.M > BM && L.N >= 128;
-    if (const char* e = std::getenv("SAMA_TC_PAIR")) pair = pair && std::atoi(e) != 0;
-    if (pair) {
-        auto ctas = [&](int w) { return 2 * (int64_t)((L.M + 2 * BM - 1) / (2 * BM)) * ((L.N + w - 1) / w) * nbr; };
-        int pbn = 0;
-        if (L.N >= 256 && ctas(256) >= ctx->sm_count) pbn = 256;
-        else if (ctas(128) >= ctx->sm_count) pbn = 128;
-        if (ctx->tile_override == 64 || ctx->tile_override == 128 || ctx->tile_override == 256) pbn = ctx->tile_override;
-        if (pbn == 0 || L.N < pbn) pair = false; else bn = pbn;
+    int bn = 64;
+    bool pair = false;
+    if (narrow_last) {
+        bn = 16;
+    } else {
+        struct Cand { int bn; bool pair; double t_kb, t_tile; };
+        const Cand cands[3] = {{64, false, 0.55, 3.0}, {128, false, 0.72, 4.0}, {256, true, 1.12, 6.0}};
+        const bool pair_ok = L.M > BM && L.N >= 256;
+        bool no_pair = false;
+        if (const char* e = std::getenv("SAMA_TC_PAIR")) no_pair = std::atoi(e) == 0;
+        double best = 0.0;
+        for (const Cand& c : cands) {
+            if (c.bn == 128 && L.N <= 64) continue;
+            if (c.pair && (!pair_ok || no_pair)) continue;
+            const int64_t tm = c.pair ? (L.M + 2 * BM - 1) / (2 * BM) : (L.M + BM - 1) / BM;
+            const int64_t items = tm * ((L.N + c.bn - 1) / c.bn) * nbr;
+            const int64_t units = c.pair ? ctx->sm_count / 2 : ctx->sm_count;
+            const double cost = (double)((items + units - 1) / units) * (num_kb * c.t_kb + c.t_tile);
+            if (best == 0.0 || cost < best) { best = cost; bn = c.bn; pair = c.pair; }
+        }
+        // override for experiments (SAMA_TC_TILE): 64 / 128 force a single-CTA width, 256 the pair
+        const int ov = ctx->tile_override;
+        if (ov == 64 || ov == 128) { bn = ov; pair = false; }
+        if (ov == 256 && pair_ok && !no_pair) { bn = 256; pair = true; }
     }
     CUtensorMap maps[4];
     const int a_slabs = (L.shared_a || nbr == 1) ? 1 : 2;
@@ -760,7 +787,7 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     a.out_lo = L.out_lo;
     a.M = L.M;
     a.N = L.N;
-    a.num_kb = Kp / BKF;
+    a.num_kb = num_kb;
     a.ldc = L.ldc;
     a.ld_next = round_up32(L.N);
     a.relu = L.relu;
@@ -783,11 +810,7 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     const int sms = ctx->sm_count;
     KernelScope scope(ctx, SAMA_K_GEMM_TF32X3, L.layer, st);
     // eight epilogue warps (two per lane quarter, each taking half of the columns) except on the 16-wide tile
-    if (pair) {
-        if (bn == 64) return launch_tc<64, true, 8>(maps, a, items, sms, st);
-        if (bn == 256) return launch_tc<256, true, 8>(maps, a, items, sms, st);
-        return launch_tc<128, true, 8>(maps, a, items, sms, st);
-    }
+    if (pair) return launch_tc<256, true, 8>(maps, a, items, sms, st);
     if (bn == 16) return launch_tc<16, false, 4>(maps, a, items, sms, st);
     if (bn == 64) return launch_tc<64, false, 8>(maps, a, items, sms, st);
     return launch_tc<128, false, 8>(maps, a, items, sms, st);
