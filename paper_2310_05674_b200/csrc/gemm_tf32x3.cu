@@ -104,6 +104,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
 // CTA-pair (cta_group::2) forms.  Shared-memory addresses of a cluster carry the CTA rank in bit 24:
 // clearing it names the same offset in the even ("leader") CTA of the pair.
 constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu;
+// The shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -226,6 +232,8 @@ struct TcArgs {
     int ldm;
     int tiles_m, tiles_n, group_n;
     int branches;          // 1 or 2; a work item is (branch, tile)
+    int ksplit;            // single-CTA tiles only: CTAs of a cluster that share one tile's contraction (1, 2 or 4)
+    float4* ws;            // ksplit > 1: partial tiles, [item][ksplit - 1][128 x BN floats]
     uint32_t tx_bytes;     // bytes the four copies of one k-block deliver
     int32_t* status;
 };
@@ -233,6 +241,9 @@ struct TcArgs {
 // Persistent kernel: CTA (or CTA pair) u of U works on tiles u, u + U, u + 2U, ... of the layer; the copy
 // pipeline and the two accumulators keep running across tiles, so the stores of one tile overlap the
 // products of the next.
+// Layers with fewer tiles than SMs can instead give one tile to a cluster of `ksplit` CTAs, each taking a
+// share of the k-blocks; the others pass their partial sums to the first through a small L2-resident
+// workspace (ordered by a cluster-scope mbarrier), and the first adds them in rank order and stores.
 // PAIR = true: two CTAs of a cluster work on one 256 x BN tile.  Each stages its own 128 rows of A and half of
 // the W tile; the leader CTA issues cta_group::2 products that read both CTAs' shared memory and write both
 // CTAs' tensor memory.  Per CTA and flop that is fewer operand bytes than two independent 128 x BN tiles.
@@ -265,7 +276,8 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
     auto acc_full_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };        // chunk in accumulator b is complete
     auto acc_empty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };   // accumulator b has been read out
-    const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 4);
+    const uint32_t part_bar = bars + 8u * (2 * STAGES + 4);   // K-split: the other CTAs' partial sums have been written
+    const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 5);
     const uint32_t abort_slot = tmem_slot + 4;
     volatile uint32_t* abort_flag =
         reinterpret_cast<volatile uint32_t*>(smem_raw + (abort_slot - smem_u32(smem_raw)));
@@ -273,12 +285,19 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;  // 0 = leader of the pair
-    const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
-    const int n_units = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const int ks = PAIR ? 1 : args.ksplit;
+    const uint32_t crank = cluster_ctarank();             // 0 without a cluster
+    const uint32_t rank = PAIR ? crank : 0u;              // 0 = leader of the pair
+    const int kpart = PAIR ? 0 : (int)crank;              // which share of the contraction
+    const int csize = PAIR ? 2 : ks;
+    const int unit = (int)blockIdx.x / csize;
+    const int n_units = (int)gridDim.x / csize;
     const int tiles_per_branch = args.tiles_m * args.tiles_n;
     const int n_items = tiles_per_branch * args.branches;
-    const int num_kb = args.num_kb;
+    // this CTA's k-blocks (the host makes every share non-empty)
+    const int kb_per_part = (args.num_kb + ks - 1) / ks;
+    const int kb_begin = kpart * kb_per_part;
+    const int num_kb = min(kb_per_part, args.num_kb - kb_begin);
     // Work item -> branch and tile origin.  Tile order inside a branch: items that run together cover all
     // M-tiles of a group of `group_n` N-tiles, so one wave re-uses a bounded set of W tiles and every A tile
     // from L2 instead of sweeping all of W.
@@ -304,6 +323,7 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
             mbar_init(acc_full_bar(b), 1);
             mbar_init(acc_empty_bar(b), EPI * (PAIR ? 2 : 1));  // one arrival per epilogue warp (of both CTAs of a pair)
         }
+        mbar_init(part_bar, EPI * (ks > 1 ? ks - 1 : 1));       // one arrival per epilogue warp of every other CTA
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -312,7 +332,7 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     }
     tc_fence_before();
     __syncthreads();
-    if (PAIR) cluster_sync();  // the peer's barriers exist before anything is signalled on them
+    if (PAIR || ks > 1) cluster_sync();  // the peer's barriers exist before anything is signalled on them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr_slot;
     // everything above (barriers, tensor memory) overlapped the previous kernel's tail; its outputs
@@ -340,7 +360,7 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (issued >= STAGES && !mbar_wait(empty_bar(s), empty_parity, abort_flag)) { raise_timeout(); ok = false; break; }
                     const uint32_t st = base + s * STAGE;
-                    const int kx = kb * BKF;
+                    const int kx = (kb_begin + kb) * BKF;
                     if (PAIR) {
                         // both CTAs' copies complete on the leader's barrier, which the leader arms for all of them
                         const uint32_t lbar = full_bar(s) & kPeerBitMask;
@@ -466,14 +486,84 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                 }
             }
             if (!ok) break;
+            if (ks > 1) {
+                // K-split: thread t of every CTA holds the same rows and columns.  Layout of a partial tile:
+                // [epilogue warp][float4 index][lane], so that a warp's accesses are contiguous.
+                float4* slab0 = args.ws + (size_t)item * (ks - 1) * (BM * BN / 4) + ((warp - 2) * (CPW / 4)) * 32 + lane;
+                if (kpart > 0) {
+                    float4* mine = slab0 + (size_t)(kpart - 1) * (BM * BN / 4);
+#pragma unroll
+                    for (int k = 0; k < CPW / 4; ++k)
+                        __stcg(mine + k * 32, make_float4(acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]));
+                    __threadfence();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(map_to_rank(part_bar, 0u));
+                    continue;  // the first CTA of the cluster finishes the tile
+                }
+                if (lane == 0) {
+                    const long long t0 = clock64();
+                    while (!mbar_try(part_bar, 0)) {   // one tile per cluster: first phase
+                        if (*abort_flag) { ok = false; break; }
+                        if (clock64() - t0 > 2 * kWaitCycles) { raise_timeout(); ok = false; break; }
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                __threadfence();
+                for (int p = 1; p < ks; ++p) {
+                    const float4* theirs = slab0 + (size_t)(p - 1) * (BM * BN / 4);
+#pragma unroll
+                    for (int k = 0; k < CPW / 4; ++k) {
+                        const float4 t = __ldcg(theirs + k * 32);
+                        acc[4 * k] += t.x; acc[4 * k + 1] += t.y; acc[4 * k + 2] += t.z; acc[4 * k + 3] += t.w;
+                    }
+                }
+            }
             // The tile's sum is in registers; the products of the next tile already run while it is stored.
-            // A thread holds one row; to store whole 128-byte row segments the warp passes each 32 x 32 block
-            // through shared memory (16-byte chunks XOR-swizzled by row: no bank conflicts either way), after
-            // which eight lanes cover one row's 32 columns and an instruction writes four full segments.
-            float4* stg = reinterpret_cast<float4*>(smem_raw + (bars + 256u - smem_u32(smem_raw))) + (warp - 2) * 256;
             const float* bias = br ? args.bias[1] : args.bias[0];
             float* outf = br ? args.out_f32[1] : args.out_f32[0];
             const bool vec_f32 = (args.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(outf) & 15u) == 0;
+            if (args.last) {
+                // fp32 output only: each thread stores its own row, 64 bytes at a time.  (Measured faster than
+                // the staged form below for this case: the staging competes with the next tile's operand
+                // fetches for shared-memory bandwidth, and there is only one output array to write.)
+                const int m = m0 + q * 32 + lane;
+                if (m < args.M) {
+#pragma unroll
+                    for (int c = 0; c < CPW; c += 16) {
+                        const int n = n0 + col0 + c;
+                        float v[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            float x = acc[c + j] + ((bias != nullptr && n + j < args.N) ? bias[n + j] : 0.f);
+                            if (args.relu && x < 0.f) x = 0.f;
+                            v[j] = x;
+                        }
+                        if (args.mask) {  // backward pass: the derivative passes only where the forward activation was positive
+                            const float* mk = args.mask + (int64_t)m * args.ldm + n;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (n + j < args.N && !(mk[j] > 0.f)) v[j] = 0.f;
+                        }
+                        float* dst = outf + (int64_t)m * args.ldc + n;
+                        if (vec_f32 && n + 15 < args.N) {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                reinterpret_cast<float4*>(dst)[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (n + j < args.N) dst[j] = v[j];
+                        }
+                    }
+                }
+                continue;
+            }
+            // Hidden layers write the next layer's hi / lo operands (and, when asked, fp32 as well).  A thread
+            // holds one row; to store whole 128-byte row segments the warp passes each 32 x 32 block through
+            // shared memory (16-byte chunks XOR-swizzled by row: no bank conflicts either way), after which
+            // eight lanes cover one row's 32 columns and an instruction writes four full segments.
+            float4* stg = reinterpret_cast<float4*>(smem_raw + (bars + 256u - smem_u32(smem_raw))) + (warp - 2) * 256;
             const int c4 = lane & 7;
 #pragma unroll
             for (int g = 0; g < ACC_REGS / 32; ++g) {
@@ -506,7 +596,7 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                             for (int j = 0; j < 4; ++j)
                                 if (n + j < args.N && !(mk[j] > 0.f)) v[j] = 0.f;
                         }
-                        if (args.last || args.both) {
+                        if (args.both) {
                             float* dst = outf + (int64_t)m * args.ldc + n;
                             if (vec_f32 && n + 3 < args.N) {
                                 *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
@@ -516,7 +606,7 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                                     if (n + j < args.N) dst[j] = v[j];
                             }
                         }
-                        if (!args.last && n < args.ld_next) {
+                        if (n < args.ld_next) {
                             // columns in [N, ld_next) are the next layer's zero padding along K
                             const int64_t off = ((int64_t)br * args.M + m) * args.ld_next + n;
                             float hi[4], lo[4];
@@ -536,7 +626,7 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     }
     tc_fence_before();
     __syncthreads();
-    if (PAIR) cluster_sync();  // neither CTA leaves (or frees tensor memory) while the other may still use it
+    if (PAIR || ks > 1) cluster_sync();  // no CTA leaves (or frees tensor memory) while another may still signal or use it
     if (warp == 1) {
         tc_fence_after();
         if (PAIR) tmem_dealloc_pair(tmem_base, TMEM_COLS); else tmem_dealloc(tmem_base, TMEM_COLS);
@@ -659,6 +749,7 @@ bool make_map(CUtensorMap* map, const float* base, int ld, int64_t rows, int sla
 // Launches the persistent kernel on min(work items, co-resident CTAs or CTA pairs) units.
 template <int BN, bool PAIR, int EPI>
 cudaError_t launch_tc(const CUtensorMap maps[4], const TcArgs& a, int items, int sm_count, cudaStream_t st) {
+    const int ks = PAIR ? 1 : a.ksplit;
     constexpr int kSmem = smem_bytes(PAIR ? BN / 2 : BN);
     static int max_units = 0;  // one CTA per SM (shared memory); pairs: what the cluster scheduler can co-schedule
     if (max_units == 0) {
@@ -686,6 +777,9 @@ cudaError_t launch_tc(const CUtensorMap maps[4], const TcArgs& a, int items, int
         if (units < 1) return cudaErrorLaunchOutOfResources;
         max_units = units;
     }
+    if (ks > 1)  // one tile per cluster of ks CTAs
+        return launch_clustered(ks, gemm_tf32x3_kernel<BN, PAIR, EPI>, dim3(items * ks), dim3(threads_for(EPI)),
+                                (size_t)kSmem, st, maps[0], maps[1], maps[2], maps[3], a);
     const int units = items < max_units ? items : max_units;
     return launch_clustered(PAIR ? 2 : 1, gemm_tf32x3_kernel<BN, PAIR, EPI>, dim3(units * (PAIR ? 2 : 1)),
                             dim3(threads_for(EPI)), (size_t)kSmem, st, maps[0], maps[1], maps[2], maps[3], a);
@@ -741,7 +835,7 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     // is taken.  Times per k-block (microseconds, measured on the three workloads): wider tiles do more
     // work per staged operand byte, narrower ones fill the machine when the layer has few tiles.
     const bool narrow_last = L.last && L.N <= 16;
-    int bn = 64;
+    int bn = 64, ksplit = 1;
     bool pair = false;
     if (narrow_last) {
         bn = 16;
@@ -759,12 +853,20 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
             const int64_t items = tm * ((L.N + c.bn - 1) / c.bn) * nbr;
             const int64_t units = c.pair ? ctx->sm_count / 2 : ctx->sm_count;
             const double cost = (double)((items + units - 1) / units) * (num_kb * c.t_kb + c.t_tile);
-            if (best == 0.0 || cost < best) { best = cost; bn = c.bn; pair = c.pair; }
+            if (best == 0.0 || cost < best) { best = cost; bn = c.bn; pair = c.pair; ksplit = 1; }
+            // a layer with few tiles: a cluster of 2 or 4 CTAs shares each tile's contraction (one wave,
+            // at least two k-blocks per CTA, about 3 us to pass the partial sums on)
+            for (int ks = 2; ks <= 4 && !c.pair && ctx->tc_ws; ks *= 2) {
+                if (items * ks > units || num_kb < 2 * ks || (size_t)items * (ks - 1) * BM * c.bn > ctx->tc_ws_floats) break;
+                const double cost_ks = ((num_kb + ks - 1) / ks) * c.t_kb + c.t_tile + 3.0;
+                if (cost_ks < best) { best = cost_ks; bn = c.bn; pair = false; ksplit = ks; }
+            }
         }
+        if (const char* e = std::getenv("SAMA_TC_KSPLIT")) { if (std::atoi(e) == 1) ksplit = 1; }
         // override for experiments (SAMA_TC_TILE): 64 / 128 force a single-CTA width, 256 the pair
         const int ov = ctx->tile_override;
-        if (ov == 64 || ov == 128) { bn = ov; pair = false; }
-        if (ov == 256 && pair_ok && !no_pair) { bn = 256; pair = true; }
+        if (ov == 64 || ov == 128) { bn = ov; pair = false; ksplit = 1; }
+        if (ov == 256 && pair_ok && !no_pair) { bn = 256; pair = true; ksplit = 1; }
     }
     CUtensorMap maps[4];
     const int a_slabs = (L.shared_a || nbr == 1) ? 1 : 2;
@@ -801,6 +903,8 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     a.tiles_m = pair ? (L.M + 2 * BM - 1) / (2 * BM) : (L.M + BM - 1) / BM;
     a.tiles_n = (L.N + bn - 1) / bn;
     a.branches = nbr;
+    a.ksplit = pair ? 1 : ksplit;
+    a.ws = reinterpret_cast<float4*>(ctx->tc_ws);
     // about one wave of CTAs per group: group_n N-tiles x all M-tiles
     a.group_n = ctx->sm_count / a.tiles_m;
     if (a.group_n < 1) a.group_n = 1;

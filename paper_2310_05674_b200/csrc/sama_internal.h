@@ -85,6 +85,8 @@ struct sama_ctx {
     float* w_split;                // device [hi, lo][2 branches][slab]: every layer's W, rows padded to 32
     float* a_split[2];             // device, ping-pong: [2][2][max_batch][round32(max hidden)]
     size_t x_split_half, w_split_half, a_split_half;  // floats per hi (or lo) part; 0 = path unavailable
+    float* tc_ws;                  // device: partial tiles of the tensor-core path's K-split (one 128 x 128 tile per SM)
+    size_t tc_ws_floats;
     float* mg_ws;                  // device: workspace of the direct gradient (activations, dz, losses)
     size_t mg_ws_floats;
     float* mg_tc;                  // device: TF32 operand buffers of the direct gradient's tensor-core path
