@@ -119,6 +119,12 @@ __device__ __forceinline__ void cluster_sync() {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// Execution barrier only.  (With release semantics every thread's arrival is a fence over the CTA's earlier
+// stores; at the end of a tile that was measured at 13-20 us.)
+__device__ __forceinline__ void cluster_sync_relaxed() {
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+}
 // Load into THIS CTA's shared memory; completion bytes are signalled on the leader's mbarrier.  No multicast.
 __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t leader_bar, int x, int y, int z) {
     asm volatile(
@@ -238,6 +244,83 @@ struct TcArgs {
     int32_t* status;
 };
 
+// Stores one 32 x 32 block of a tile that a warp has laid out in shared memory (`stg`: 32 rows of eight
+// 16-byte chunks, chunk c of row r at position c ^ (r & 7)).  Eight lanes cover one row's 32 columns, so an
+// instruction writes four full 128-byte segments.  Adds the bias, applies ReLU and the mask, and writes fp32
+// and / or the next layer's hi / lo operands.  Deliberately not inlined and not unrolled: it runs once per
+// block, and straight-line code that is executed once costs more in instruction fetches than it saves.
+__device__ __noinline__ void store_block(const TcArgs& args, const float4* stg, int br, int m_base, int n_base,
+                                         int valid_cols, int lane) {
+    const int c4 = lane & 7;
+    if (4 * c4 >= valid_cols) return;  // (the 16-wide tile fills only half of the block)
+    const int n = n_base + 4 * c4;
+    const int N = args.N;
+    const int r0 = lane >> 3;          // this lane's rows of the block: r0, r0 + 4, ..., r0 + 28
+    const int rows = min(32, args.M - m_base);
+    const float* bias = br ? args.bias[1] : args.bias[0];
+    float* outf = br ? args.out_f32[1] : args.out_f32[0];
+    const bool want_f32 = args.last || args.both;
+    const bool want_split = !args.last && n < args.ld_next;
+    const bool relu = args.relu != 0;
+    const bool full = n + 3 < N;       // all four columns exist
+    const bool vec_f32 = full && (args.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(outf) & 15u) == 0;
+    float b[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) b[j] = (bias != nullptr && n + j < N) ? bias[n + j] : 0.f;
+    // everything that depends on the row advances by a fixed stride (4 rows) per iteration
+    const int64_t row0 = (int64_t)m_base + r0;
+    const float* mk = args.mask ? args.mask + row0 * args.ldm + n : nullptr;
+    float* dst = outf + row0 * args.ldc + n;
+    float* dh = args.out_hi + ((int64_t)br * args.M + row0) * args.ld_next + n;
+    float* dl = args.out_lo + ((int64_t)br * args.M + row0) * args.ld_next + n;
+    const int64_t mk_step = 4 * (int64_t)args.ldm, dst_step = 4 * (int64_t)args.ldc, split_step = 4 * (int64_t)args.ld_next;
+    // chunk position of this lane's columns in rows r0 + 8 j and in rows r0 + 4 + 8 j
+    const float4* src_even = stg + r0 * 8 + (c4 ^ r0);
+    const float4* src_odd = stg + (r0 + 4) * 8 + (c4 ^ (r0 + 4));
+#pragma unroll 2
+    for (int i = 0; i < 8; ++i) {
+        const int rl = r0 + 4 * i;
+        if (rl < rows) {
+            const float4 t = ((i & 1) ? src_odd : src_even)[(i >> 1) * 64];
+            float v[4] = {t.x + b[0], t.y + b[1], t.z + b[2], t.w + b[3]};
+            if (relu) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) v[j] = fmaxf(v[j], 0.f);
+            }
+            if (mk) {  // backward pass: the derivative passes only where the forward activation was positive
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (n + j < N && !(mk[j] > 0.f)) v[j] = 0.f;
+            }
+            if (want_f32) {
+                if (vec_f32) {
+                    *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (n + j < N) dst[j] = v[j];
+                }
+            }
+            if (want_split) {
+                // columns in [N, ld_next) are the next layer's zero padding along K
+                float hi[4], lo[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float x = (full || n + j < N) ? v[j] : 0.f;
+                    hi[j] = to_tf32(x);
+                    lo[j] = to_tf32(x - hi[j]);
+                }
+                *reinterpret_cast<float4*>(dh) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<float4*>(dl) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+            }
+        }
+        if (mk) mk += mk_step;
+        dst += dst_step;
+        dh += split_step;
+        dl += split_step;
+    }
+}
+
 // Persistent kernel: CTA (or CTA pair) u of U works on tiles u, u + U, u + 2U, ... of the layer; the copy
 // pipeline and the two accumulators keep running across tiles, so the stores of one tile overlap the
 // products of the next.
@@ -251,7 +334,7 @@ template <int BN, bool PAIR, int EPI>
 __global__ void __launch_bounds__(threads_for(EPI), 1)
 gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
                    const __grid_constant__ CUtensorMap map_w_hi, const __grid_constant__ CUtensorMap map_w_lo,
-                   TcArgs args) {
+                   const __grid_constant__ TcArgs args) {
     constexpr int WROWS = PAIR ? BN / 2 : BN;  // rows of W this CTA stages
     constexpr int STAGES = stages_for(WROWS);
     constexpr int A_BYTES = BM * BKF * 4, W_BYTES = WROWS * BKF * 4;
@@ -443,6 +526,8 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         const int col0 = ((warp - 2) >> 2) * CPW;  // with eight epilogue warps, two share a lane quarter and split the columns
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)col0;
         const int n_chunks = (num_kb + kChunkKb - 1) / kChunkKb;
+        const int my_items = unit < n_items ? (n_items - unit + n_units - 1) / n_units : 0;
+        const int total_chunks = my_items * n_chunks;
         int chunk = 0;  // counts over all of this CTA's tiles, like the issuer's
         bool ok = true;
         for (int item = unit; item < n_items && ok; item += n_units) {
@@ -481,7 +566,9 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                 // this warp's reads are done: hand the accumulator back to the MMA issuer
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) {
+                // (not for the last two chunks: nobody waits for them, and no arrival on the peer's barrier may
+                // still be on its way when that CTA exits)
+                if (lane == 0 && chunk + 2 < total_chunks) {
                     if (PAIR) mbar_arrive_cluster(acc_empty_bar(buf) & kPeerBitMask); else mbar_arrive(acc_empty_bar(buf));
                 }
             }
@@ -520,51 +607,9 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                 }
             }
             // The tile's sum is in registers; the products of the next tile already run while it is stored.
-            const float* bias = br ? args.bias[1] : args.bias[0];
-            float* outf = br ? args.out_f32[1] : args.out_f32[0];
-            const bool vec_f32 = (args.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(outf) & 15u) == 0;
-            if (args.last) {
-                // fp32 output only: each thread stores its own row, 64 bytes at a time.  (Measured faster than
-                // the staged form below for this case: the staging competes with the next tile's operand
-                // fetches for shared-memory bandwidth, and there is only one output array to write.)
-                const int m = m0 + q * 32 + lane;
-                if (m < args.M) {
-#pragma unroll
-                    for (int c = 0; c < CPW; c += 16) {
-                        const int n = n0 + col0 + c;
-                        float v[16];
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            float x = acc[c + j] + ((bias != nullptr && n + j < args.N) ? bias[n + j] : 0.f);
-                            if (args.relu && x < 0.f) x = 0.f;
-                            v[j] = x;
-                        }
-                        if (args.mask) {  // backward pass: the derivative passes only where the forward activation was positive
-                            const float* mk = args.mask + (int64_t)m * args.ldm + n;
-#pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                if (n + j < args.N && !(mk[j] > 0.f)) v[j] = 0.f;
-                        }
-                        float* dst = outf + (int64_t)m * args.ldc + n;
-                        if (vec_f32 && n + 15 < args.N) {
-#pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                reinterpret_cast<float4*>(dst)[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                if (n + j < args.N) dst[j] = v[j];
-                        }
-                    }
-                }
-                continue;
-            }
-            // Hidden layers write the next layer's hi / lo operands (and, when asked, fp32 as well).  A thread
-            // holds one row; to store whole 128-byte row segments the warp passes each 32 x 32 block through
-            // shared memory (16-byte chunks XOR-swizzled by row: no bank conflicts either way), after which
-            // eight lanes cover one row's 32 columns and an instruction writes four full segments.
+            // A thread holds one row; to store whole 128-byte row segments the warp passes each 32 x 32 block
+            // through shared memory (16-byte chunks XOR-swizzled by row: no bank conflicts either way).
             float4* stg = reinterpret_cast<float4*>(smem_raw + (bars + 256u - smem_u32(smem_raw))) + (warp - 2) * 256;
-            const int c4 = lane & 7;
 #pragma unroll
             for (int g = 0; g < ACC_REGS / 32; ++g) {
                 __syncwarp();
@@ -573,60 +618,15 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                     stg[lane * 8 + (k ^ (lane & 7))] =
                         make_float4(acc[32 * g + 4 * k], acc[32 * g + 4 * k + 1], acc[32 * g + 4 * k + 2], acc[32 * g + 4 * k + 3]);
                 __syncwarp();
-                const int cl = 32 * g + 4 * c4;  // this lane's four columns within the thread's column range
-                const int n = n0 + col0 + cl;
-                if (cl < CPW) {                  // (the 16-wide tile fills only half of the block)
-                    float b[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) b[j] = (bias != nullptr && n + j < args.N) ? bias[n + j] : 0.f;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int rl = 4 * i + (lane >> 3);
-                        const int m = m0 + q * 32 + rl;
-                        const float4 t = stg[rl * 8 + (c4 ^ (rl & 7))];
-                        if (m >= args.M) continue;
-                        float v[4] = {t.x + b[0], t.y + b[1], t.z + b[2], t.w + b[3]};
-                        if (args.relu) {
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) v[j] = v[j] < 0.f ? 0.f : v[j];
-                        }
-                        if (args.mask) {  // backward pass: the derivative passes only where the forward activation was positive
-                            const float* mk = args.mask + (int64_t)m * args.ldm + n;
-#pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                if (n + j < args.N && !(mk[j] > 0.f)) v[j] = 0.f;
-                        }
-                        if (args.both) {
-                            float* dst = outf + (int64_t)m * args.ldc + n;
-                            if (vec_f32 && n + 3 < args.N) {
-                                *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 4; ++j)
-                                    if (n + j < args.N) dst[j] = v[j];
-                            }
-                        }
-                        if (n < args.ld_next) {
-                            // columns in [N, ld_next) are the next layer's zero padding along K
-                            const int64_t off = ((int64_t)br * args.M + m) * args.ld_next + n;
-                            float hi[4], lo[4];
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const float x = (n + j < args.N) ? v[j] : 0.f;
-                                hi[j] = to_tf32(x);
-                                lo[j] = to_tf32(x - hi[j]);
-                            }
-                            *reinterpret_cast<float4*>(args.out_hi + off) = make_float4(hi[0], hi[1], hi[2], hi[3]);
-                            *reinterpret_cast<float4*>(args.out_lo + off) = make_float4(lo[0], lo[1], lo[2], lo[3]);
-                        }
-                    }
-                }
+                store_block(args, stg, br, m0 + q * 32, n0 + col0 + 32 * g, CPW - 32 * g, lane);
             }
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (PAIR || ks > 1) cluster_sync();  // no CTA leaves (or frees tensor memory) while another may still signal or use it
+    // A pair leaves together: the leader's products use the peer's shared and tensor memory.  (K-split CTAs
+    // may leave on their own: the only remote access is the arrival that the first CTA has waited for.)
+    if (PAIR) cluster_sync_relaxed();
     if (warp == 1) {
         tc_fence_after();
         if (PAIR) tmem_dealloc_pair(tmem_base, TMEM_COLS); else tmem_dealloc(tmem_base, TMEM_COLS);
