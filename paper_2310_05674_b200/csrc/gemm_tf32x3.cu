@@ -225,6 +225,13 @@ __device__ __forceinline__ float to_tf32(float x) {
     return __uint_as_float(r);
 }
 
+// Round-to-nearest (ties away from zero) to TF32 with integer arithmetic: same result as cvt.rna.tf32.f32 on
+// finite values, at the full integer rate (the conversion instruction issues at a fraction of it, which shows
+// in the epilogue, where eight warps convert a whole tile).
+__device__ __forceinline__ float round_tf32(float x) {
+    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);
+}
+
 struct TcArgs {
     const float* bias[2];  // [N] fp32 (slices of theta+ / theta-), may be unaligned
     float* out_f32[2];     // fp32 output (logits, or activations feeding a fused head): [M][ldc]
@@ -247,9 +254,8 @@ struct TcArgs {
 // Stores one 32 x 32 block of a tile that a warp has laid out in shared memory (`stg`: 32 rows of eight
 // 16-byte chunks, chunk c of row r at position c ^ (r & 7)).  Eight lanes cover one row's 32 columns, so an
 // instruction writes four full 128-byte segments.  Adds the bias, applies ReLU and the mask, and writes fp32
-// and / or the next layer's hi / lo operands.  Deliberately not inlined and not unrolled: it runs once per
-// block, and straight-line code that is executed once costs more in instruction fetches than it saves.
-__device__ __noinline__ void store_block(const TcArgs& args, const float4* stg, int br, int m_base, int n_base,
+// and / or the next layer's hi / lo operands.
+__device__ __forceinline__ void store_block(const TcArgs& args, const float4* stg, int br, int m_base, int n_base,
                                          int valid_cols, int lane) {
     const int c4 = lane & 7;
     if (4 * c4 >= valid_cols) return;  // (the 16-wide tile fills only half of the block)
@@ -277,28 +283,49 @@ __device__ __noinline__ void store_block(const TcArgs& args, const float4* stg, 
     // chunk position of this lane's columns in rows r0 + 8 j and in rows r0 + 4 + 8 j
     const float4* src_even = stg + r0 * 8 + (c4 ^ r0);
     const float4* src_odd = stg + (r0 + 4) * 8 + (c4 ^ (r0 + 4));
-#pragma unroll 2
+    // all eight rows are fetched first (rows beyond M hold stale data that is never stored), so that the
+    // eight independent chains of arithmetic and stores can overlap
+    float4 t[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) t[i] = ((i & 1) ? src_odd : src_even)[(i >> 1) * 64];
+    const float floor_v = relu ? 0.f : -3.402823466e38f;  // max(x, floor_v): ReLU or (for finite x) nothing
+    if (full && rows == 32 && mk == nullptr && (vec_f32 || !want_f32)) {
+        // interior block: no per-row or per-column conditions (branches cost more here than the arithmetic)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float v0 = fmaxf(t[i].x + b[0], floor_v), v1 = fmaxf(t[i].y + b[1], floor_v);
+            const float v2 = fmaxf(t[i].z + b[2], floor_v), v3 = fmaxf(t[i].w + b[3], floor_v);
+            if (want_f32) *reinterpret_cast<float4*>(dst + i * dst_step) = make_float4(v0, v1, v2, v3);
+            if (want_split) {
+                const float h0 = round_tf32(v0), h1 = round_tf32(v1), h2 = round_tf32(v2), h3 = round_tf32(v3);
+                *reinterpret_cast<float4*>(dh + i * split_step) = make_float4(h0, h1, h2, h3);
+                *reinterpret_cast<float4*>(dl + i * split_step) =
+                    make_float4(round_tf32(v0 - h0), round_tf32(v1 - h1), round_tf32(v2 - h2), round_tf32(v3 - h3));
+            }
+        }
+        return;
+    }
+#pragma unroll 1
     for (int i = 0; i < 8; ++i) {
         const int rl = r0 + 4 * i;
         if (rl < rows) {
-            const float4 t = ((i & 1) ? src_odd : src_even)[(i >> 1) * 64];
-            float v[4] = {t.x + b[0], t.y + b[1], t.z + b[2], t.w + b[3]};
-            if (relu) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) v[j] = fmaxf(v[j], 0.f);
-            }
+            const float4 ti = ((i & 1) ? src_odd : src_even)[(i >> 1) * 64];
+            float v[4] = {fmaxf(ti.x + b[0], floor_v), fmaxf(ti.y + b[1], floor_v), fmaxf(ti.z + b[2], floor_v),
+                          fmaxf(ti.w + b[3], floor_v)};
             if (mk) {  // backward pass: the derivative passes only where the forward activation was positive
+                const float* mrow = mk + i * mk_step;
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
-                    if (n + j < N && !(mk[j] > 0.f)) v[j] = 0.f;
+                    if (n + j < N && !(mrow[j] > 0.f)) v[j] = 0.f;
             }
             if (want_f32) {
+                float* drow = dst + i * dst_step;
                 if (vec_f32) {
-                    *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+                    *reinterpret_cast<float4*>(drow) = make_float4(v[0], v[1], v[2], v[3]);
                 } else {
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
-                        if (n + j < N) dst[j] = v[j];
+                        if (n + j < N) drow[j] = v[j];
                 }
             }
             if (want_split) {
@@ -307,17 +334,13 @@ __device__ __noinline__ void store_block(const TcArgs& args, const float4* stg, 
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const float x = (full || n + j < N) ? v[j] : 0.f;
-                    hi[j] = to_tf32(x);
-                    lo[j] = to_tf32(x - hi[j]);
+                    hi[j] = round_tf32(x);
+                    lo[j] = round_tf32(x - hi[j]);
                 }
-                *reinterpret_cast<float4*>(dh) = make_float4(hi[0], hi[1], hi[2], hi[3]);
-                *reinterpret_cast<float4*>(dl) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                *reinterpret_cast<float4*>(dh + i * split_step) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<float4*>(dl + i * split_step) = make_float4(lo[0], lo[1], lo[2], lo[3]);
             }
         }
-        if (mk) mk += mk_step;
-        dst += dst_step;
-        dh += split_step;
-        dl += split_step;
     }
 }
 
@@ -855,10 +878,11 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
             const double cost = (double)((items + units - 1) / units) * (num_kb * c.t_kb + c.t_tile);
             if (best == 0.0 || cost < best) { best = cost; bn = c.bn; pair = c.pair; ksplit = 1; }
             // a layer with few tiles: a cluster of 2 or 4 CTAs shares each tile's contraction (one wave,
-            // at least two k-blocks per CTA, about 3 us to pass the partial sums on)
+            // at least two k-blocks per CTA, about 6 us to pass the partial sums on and for the first CTA to
+            // store the whole tile alone)
             for (int ks = 2; ks <= 4 && !c.pair && ctx->tc_ws; ks *= 2) {
                 if (items * ks > units || num_kb < 2 * ks || (size_t)items * (ks - 1) * BM * c.bn > ctx->tc_ws_floats) break;
-                const double cost_ks = ((num_kb + ks - 1) / ks) * c.t_kb + c.t_tile + 3.0;
+                const double cost_ks = ((num_kb + ks - 1) / ks) * c.t_kb + c.t_tile + 6.0;
                 if (cost_ks < best) { best = cost_ks; bn = c.bn; pair = false; ksplit = ks; }
             }
         }
