@@ -246,7 +246,7 @@ struct TcArgs {
     int tiles_m, tiles_n, group_n;
     int branches;          // 1 or 2; a work item is (branch, tile)
     int ksplit;            // single-CTA tiles only: CTAs of a cluster that share one tile's contraction (1, 2 or 4)
-    float4* ws;            // ksplit > 1: partial tiles, [item][ksplit - 1][128 x BN floats]
+    float4* ws;            // ksplit > 1: partial tiles, [item][ksplit][128 x BN floats]
     uint32_t tx_bytes;     // bytes the four copies of one k-block deliver
     int32_t* status;
 };
@@ -348,8 +348,8 @@ __device__ __forceinline__ void store_block(const TcArgs& args, const float4* st
 // pipeline and the two accumulators keep running across tiles, so the stores of one tile overlap the
 // products of the next.
 // Layers with fewer tiles than SMs can instead give one tile to a cluster of `ksplit` CTAs, each taking a
-// share of the k-blocks; the others pass their partial sums to the first through a small L2-resident
-// workspace (ordered by a cluster-scope mbarrier), and the first adds them in rank order and stores.
+// share of the k-blocks; the CTAs then exchange partial sums through a small L2-resident workspace (ordered
+// by cluster-scope mbarriers) so that each adds up, in rank order, and stores an equal share of the columns.
 // PAIR = true: two CTAs of a cluster work on one 256 x BN tile.  Each stages its own 128 rows of A and half of
 // the W tile; the leader CTA issues cta_group::2 products that read both CTAs' shared memory and write both
 // CTAs' tensor memory.  Per CTA and flop that is fewer operand bytes than two independent 128 x BN tiles.
@@ -597,20 +597,26 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
             }
             if (!ok) break;
             if (ks > 1) {
-                // K-split: thread t of every CTA holds the same rows and columns.  Layout of a partial tile:
-                // [epilogue warp][float4 index][lane], so that a warp's accesses are contiguous.
-                float4* slab0 = args.ws + (size_t)item * (ks - 1) * (BM * BN / 4) + ((warp - 2) * (CPW / 4)) * 32 + lane;
-                if (kpart > 0) {
-                    float4* mine = slab0 + (size_t)(kpart - 1) * (BM * BN / 4);
+                // K-split: thread t of every CTA of the cluster holds partial sums of the same rows and columns.
+                // The tile's columns are dealt out in ks equal shares; for every 32-column block that another
+                // CTA owns, this thread leaves its partial sums in its own slab of the workspace, then the
+                // owner adds the slabs in rank order and stores its share (so all CTAs store, not just one).
+                // Layout of a slab: [epilogue warp][float4 index][lane]: a warp's accesses are contiguous.
+                const int share = BN / ks;  // >= 32 columns
+                float4* slabs = args.ws + (size_t)item * ks * (BM * BN / 4) + ((warp - 2) * (CPW / 4)) * 32 + lane;
+                float4* mine = slabs + (size_t)kpart * (BM * BN / 4);
 #pragma unroll
-                    for (int k = 0; k < CPW / 4; ++k)
+                for (int g = 0; g < CPW / 32; ++g) {
+                    if ((col0 + 32 * g) / share == kpart) continue;
+#pragma unroll
+                    for (int k = 8 * g; k < 8 * g + 8; ++k)
                         __stcg(mine + k * 32, make_float4(acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]));
-                    __threadfence();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(map_to_rank(part_bar, 0u));
-                    continue;  // the first CTA of the cluster finishes the tile
                 }
+                __threadfence();
+                __syncwarp();
                 if (lane == 0) {
+                    for (int p = 0; p < ks; ++p)
+                        if (p != kpart) mbar_arrive_cluster(map_to_rank(part_bar, (uint32_t)p));
                     const long long t0 = clock64();
                     while (!mbar_try(part_bar, 0)) {   // one tile per cluster: first phase
                         if (*abort_flag) { ok = false; break; }
@@ -620,12 +626,17 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) break;
                 __threadfence();
-                for (int p = 1; p < ks; ++p) {
-                    const float4* theirs = slab0 + (size_t)(p - 1) * (BM * BN / 4);
 #pragma unroll
-                    for (int k = 0; k < CPW / 4; ++k) {
-                        const float4 t = __ldcg(theirs + k * 32);
-                        acc[4 * k] += t.x; acc[4 * k + 1] += t.y; acc[4 * k + 2] += t.z; acc[4 * k + 3] += t.w;
+                for (int g = 0; g < CPW / 32; ++g) {
+                    if ((col0 + 32 * g) / share != kpart) continue;
+                    for (int p = 0; p < ks; ++p) {
+                        if (p == kpart) continue;
+                        const float4* theirs = slabs + (size_t)p * (BM * BN / 4);
+#pragma unroll
+                        for (int k = 8 * g; k < 8 * g + 8; ++k) {
+                            const float4 t = __ldcg(theirs + k * 32);
+                            acc[4 * k] += t.x; acc[4 * k + 1] += t.y; acc[4 * k + 2] += t.z; acc[4 * k + 3] += t.w;
+                        }
                     }
                 }
             }
@@ -641,6 +652,7 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                     stg[lane * 8 + (k ^ (lane & 7))] =
                         make_float4(acc[32 * g + 4 * k], acc[32 * g + 4 * k + 1], acc[32 * g + 4 * k + 2], acc[32 * g + 4 * k + 3]);
                 __syncwarp();
+                if (ks > 1 && (col0 + 32 * g) / (BN / ks) != kpart) continue;  // another CTA of the cluster stores this block
                 store_block(args, stg, br, m0 + q * 32, n0 + col0 + 32 * g, CPW - 32 * g, lane);
             }
         }
@@ -878,11 +890,12 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
             const double cost = (double)((items + units - 1) / units) * (num_kb * c.t_kb + c.t_tile);
             if (best == 0.0 || cost < best) { best = cost; bn = c.bn; pair = c.pair; ksplit = 1; }
             // a layer with few tiles: a cluster of 2 or 4 CTAs shares each tile's contraction (one wave,
-            // at least two k-blocks per CTA, about 6 us to pass the partial sums on and for the first CTA to
-            // store the whole tile alone)
+            // at least two k-blocks per CTA, about 4 us for the exchange; each CTA stores 1 / ks of the tile)
             for (int ks = 2; ks <= 4 && !c.pair && ctx->tc_ws; ks *= 2) {
-                if (items * ks > units || num_kb < 2 * ks || (size_t)items * (ks - 1) * BM * c.bn > ctx->tc_ws_floats) break;
-                const double cost_ks = ((num_kb + ks - 1) / ks) * c.t_kb + c.t_tile + 6.0;
+                if (items * ks > units || num_kb < 2 * ks || c.bn / ks < 32 ||
+                    (size_t)items * ks * BM * c.bn > ctx->tc_ws_floats)
+                    break;
+                const double cost_ks = ((num_kb + ks - 1) / ks) * c.t_kb + c.t_tile / ks + 4.0;
                 if (cost_ks < best) { best = cost_ks; bn = c.bn; pair = false; ksplit = ks; }
             }
         }
