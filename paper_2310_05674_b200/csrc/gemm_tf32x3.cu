@@ -9,22 +9,27 @@
 // forward passes by 2 eps_fd, which amplifies rounding by 1/eps_fd; plain TF32
 // (2^-11) would drown the signal, which is why the split is needed.
 //
-// Structure of gemm_tf32x3_kernel (one 128 x BN output tile per CTA, or one 256 x BN tile per CTA
-// pair; 2 + 4 or 2 + 8 warps):
+// Structure of gemm_tf32x3_kernel (persistent: a CTA, or a CTA pair, walks several 128 x BN, or
+// 256 x 256, output tiles of both branches; 2 + 4 or 2 + 8 warps):
 //   warp 0    : TMA producer.  Per k-block of 32 floats it loads four tiles
 //               (A hi/lo: 128 x 32, W hi/lo: BN x 32) with cp.async.bulk.tensor
 //               into 128-byte-swizzled shared memory and signals a "full"
 //               mbarrier with the byte count.  No multicast.
 //   warp 1    : allocates tensor memory (two accumulators), then one lane issues,
-//               per k-block, 4 k-steps x 3 tcgen05.mma kind::tf32 (M = 128 or 256,
-//               N = BN, K = 8) from shared-memory descriptors and commits to the
+//               per k-block, 4 k-steps of tcgen05.mma kind::tf32 (K = 8) from
+//               shared-memory descriptors -- three products per k-step, or two
+//               wider ones on single-CTA tiles (see CONCAT) -- and commits to the
 //               stage's "empty" mbarrier; every few k-blocks it commits the chunk's
-//               accumulator and moves to the other one.
+//               accumulator and moves to the other one.  The pipeline keeps running
+//               across tile boundaries.
 //   warps 2.. : epilogue.  Each warp reads its 32 lanes of a finished chunk with
 //               tcgen05.ld and adds it to a running fp32 sum in registers (the
 //               tensor core's own accumulation rounds toward zero, see kChunkKb);
-//               after the last chunk it adds the bias, applies ReLU, and either
-//               stores fp32 results or the next layer's hi/lo operands directly.
+//               after a tile's last chunk it adds the bias, applies ReLU, and stores
+//               fp32 results and / or the next layer's hi/lo operands through a
+//               shared-memory transpose, while the next tile is being multiplied.
+// A layer with fewer tiles than SMs gives each tile to a cluster of 2 or 4 CTAs that split the
+// contraction and exchange partial sums (see ksplit).
 // Operands are K-major in global memory ([rows][K], K padded to a multiple of
 // 32 with zeros), which is what both TMA and the K-major UMMA descriptor want.
 // Every mbarrier wait is bounded: if one expires the CTA raises
