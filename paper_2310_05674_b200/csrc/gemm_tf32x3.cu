@@ -955,6 +955,9 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     const int items = a.tiles_m * a.tiles_n * nbr;
     const int sms = ctx->sm_count;
     KernelScope scope(ctx, SAMA_K_GEMM_TF32X3, L.layer, st);
+    // The matrix products keep the dependent-launch overlap even inside a chain that switched it off for
+    // its small kernels (the direct gradient, see run_meta_grad_tc).
+    PdlScope pdl(pdl_enabled() ? 1 : 0);
     // eight epilogue warps (two per lane quarter, each taking half of the columns) except on the 16-wide tile
     if (pair) return launch_tc<256, true, 8>(maps, a, items, sms, st);
     if (bn == 16) return launch_tc<16, false, 4>(maps, a, items, sms, st);

@@ -320,6 +320,7 @@ int run_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const 
 }  // namespace
 
 namespace sama {
+thread_local int pdl_override = -1;
 bool pdl_enabled() {
     static const bool on = []() { const char* e = std::getenv("SAMA_NO_PDL"); return !(e && e[0] == '1'); }();
     return on;

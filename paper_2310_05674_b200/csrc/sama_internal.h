@@ -132,6 +132,14 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 #endif
 bool pdl_enabled();
+extern thread_local int pdl_override;  // -1: follow pdl_enabled(); 0 / 1: force off / on for the launches that follow
+struct PdlScope {  // sets pdl_override for the lifetime of the object
+    int old;
+    explicit PdlScope(int v) : old(pdl_override) { pdl_override = v; }
+    ~PdlScope() { pdl_override = old; }
+    PdlScope(const PdlScope&) = delete;
+    PdlScope& operator=(const PdlScope&) = delete;
+};
 template <typename... KArgs, typename... Args>
 cudaError_t launch_clustered(int cluster_x, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
                              cudaStream_t st, Args&&... args) {
@@ -149,7 +157,7 @@ cudaError_t launch_clustered(int cluster_x, void (*kernel)(KArgs...), dim3 grid,
         attr[na].val.clusterDim.z = 1;
         ++na;
     }
-    if (pdl_enabled()) {
+    if (pdl_override >= 0 ? pdl_override != 0 : pdl_enabled()) {
         attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[na].val.programmaticStreamSerializationAllowed = 1;
         ++na;
