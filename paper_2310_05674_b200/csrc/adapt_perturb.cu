@@ -326,8 +326,10 @@ perturb_split_kernel(int64_t n, const float* theta, const float* __restrict__ p,
     auto emit = [&](int64_t i, float4 vt, float4 vp) {
         float4 a, b;
         plus_minus(eps, vt, vp, a, b);
-        tp4[i] = a;
-        tm4[i] = b;
+        // theta+- themselves are not read again by the forward (only their biases and a narrow head are):
+        // streaming stores keep them from displacing the hi / lo operands, which the next kernel reads, in L2
+        __stcs(tp4 + i, a);
+        __stcs(tm4 + i, b);
         const int64_t e = i << 2;
         int l = -1;
 #pragma unroll 1
