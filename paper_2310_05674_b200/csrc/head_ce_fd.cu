@@ -2,7 +2,7 @@
 //
 // When the last layer has few outputs (C <= 16: the 10- and 4-class workloads)
 // a tiled matrix product wastes almost all of its tile, and the logits would
-// make a round trip through HBM only to be read once.  Here WPS warps (8 for
+// make a round trip through HBM only to be read once.  Here WPS warps (4 or 2 for
 // small batches, so that the dependent-load chain is short and the grid still
 // fills the machine; 1 for large batches) own one sample for BOTH branches:
 // their threads split the contraction index, each thread accumulates the C
@@ -143,15 +143,19 @@ cudaError_t launch_head_ce_fd(sama_ctx* ctx, const float* h_plus, const float* h
     const bool vec = (K % 4 == 0) && (ldh % 4 == 0) && aligned16(h_plus) && aligned16(h_minus) &&
                      aligned16(w_plus) && aligned16(w_minus);
     // a whole block per sample while that still gives every SM a few blocks; a warp per sample beyond
-    const bool wide = (int64_t)B <= 8 * (int64_t)ctx->sm_count;
-    const int grid = wide ? B : (B + kWarps - 1) / kWarps;
+    // warps per sample: more of them shorten each thread's chain of dependent loads, fewer give each block
+    // more samples to reuse the head's weights from L1 (measured: 4 is best up to B = 8 #SM, 2 up to 32 #SM)
+    const int64_t sms = ctx->sm_count;
+    const int wps = (int64_t)B <= 8 * sms ? 4 : ((int64_t)B <= 32 * sms ? 2 : 1);
+    const int spb = kWarps / wps;
+    const int grid = (B + spb - 1) / spb;
     KernelScope scope(ctx, SAMA_K_HEAD, -1, st);
     cudaError_t err = cudaSuccess;
 #define SAMA_HEAD2(CT, V, W)                                                                                       \
     err = launch_dependent(head_ce_fd_kernel<CT, V, W>, dim3(grid), dim3(kWarps * 32), 0, st, h_plus, h_minus, ldh, \
                            w_plus, w_minus, b_plus, b_minus, y, lambda, B, C, K, eps_fd, metagrad, loss_plus,      \
                            loss_minus, ctx->scalars)
-#define SAMA_HEAD(CT, V) do { if (wide) SAMA_HEAD2(CT, V, 8); else SAMA_HEAD2(CT, V, 1); } while (0)
+#define SAMA_HEAD(CT, V) do { if (wps == 4) SAMA_HEAD2(CT, V, 4); else if (wps == 2) SAMA_HEAD2(CT, V, 2); else SAMA_HEAD2(CT, V, 1); } while (0)
     if (C <= 4) { if (vec) SAMA_HEAD(4, true); else SAMA_HEAD(4, false); }
     else if (C <= 10) { if (vec) SAMA_HEAD(10, true); else SAMA_HEAD(10, false); }
     else { if (vec) SAMA_HEAD(16, true); else SAMA_HEAD(16, false); }
