@@ -109,6 +109,19 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
 // CTA-pair (cta_group::2) forms.  Shared-memory addresses of a cluster carry the CTA rank in bit 24:
 // clearing it names the same offset in the even ("leader") CTA of the pair.
 constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu;
+// try_wait whose success also makes another CTA's earlier writes (released at cluster scope) visible
+__device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void st_cluster_f4(uint32_t addr, float a, float b, float c, float d) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
 // The shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster.
 __device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
     uint32_t r;
@@ -425,6 +438,12 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         n0 = tile_n * BN;
     };
 
+    if (threadIdx.x == 32) {  // descriptor fetches off the first copies' critical path
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a_hi) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a_lo) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w_hi) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w_lo) : "memory");
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar(s), 1);
@@ -608,7 +627,45 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                 // owner adds the slabs in rank order and stores its share (so all CTAs store, not just one).
                 // Layout of a slab: [epilogue warp][float4 index][lane]: a warp's accesses are contiguous.
                 const int share = BN / ks;  // >= 32 columns
-                float4* slabs = args.ws + (size_t)item * ks * (BM * BN / 4) + ((warp - 2) * (CPW / 4)) * 32 + lane;
+                const uint32_t stage_u32 = bars + 256u;  // the warps' store-staging blocks, 4 KB each
+                const int wi = warp - 2;
+                if (EPI == 8 && ks == 2) {
+                    // Two CTAs: a warp's columns all belong to one of them (CPW = BN / 2), so in each CTA four
+                    // warps send and four receive.  The partials go straight into the receiving CTA's staging
+                    // blocks through distributed shared memory (the receiver's own block and that of its
+                    // sending neighbour, which is idle): no round trip through L2, no device-scope fences.
+                    const bool sender = (wi >> 2) != kpart;
+                    if (sender) {
+                        const uint32_t remote = map_to_rank(stage_u32, (uint32_t)(kpart ^ 1));
+#pragma unroll
+                        for (int k = 0; k < CPW / 4; ++k) {
+                            const int slot = k < 8 ? wi : (wi ^ 4);
+                            st_cluster_f4(remote + (uint32_t)slot * kStoreStageBytes + (uint32_t)(((k & 7) * 32 + lane) * 16),
+                                          acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]);
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive_cluster(map_to_rank(part_bar, (uint32_t)(kpart ^ 1)));
+                        const long long t0 = clock64();
+                        while (!mbar_try_cluster(part_bar, 0)) {   // one tile per cluster: first phase
+                            if (*abort_flag) { ok = false; break; }
+                            if (clock64() - t0 > 2 * kWaitCycles) { raise_timeout(); ok = false; break; }
+                        }
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) break;
+                    if (!sender) {
+                        const float4* blocks = reinterpret_cast<const float4*>(smem_raw + (stage_u32 - smem_u32(smem_raw)));
+#pragma unroll
+                        for (int k = 0; k < CPW / 4; ++k) {
+                            const int slot = k < 8 ? wi : (wi ^ 4);
+                            const float4 t = blocks[slot * 256 + (k & 7) * 32 + lane];
+                            acc[4 * k] += t.x; acc[4 * k + 1] += t.y; acc[4 * k + 2] += t.z; acc[4 * k + 3] += t.w;
+                        }
+                    }
+                } else {
+                float4* slabs = args.ws + (size_t)item * ks * (BM * BN / 4) + (wi * (CPW / 4)) * 32 + lane;
                 float4* mine = slabs + (size_t)kpart * (BM * BN / 4);
 #pragma unroll
                 for (int g = 0; g < CPW / 32; ++g) {
@@ -644,6 +701,7 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                         }
                     }
                 }
+                }
             }
             // The tile's sum is in registers; the products of the next tile already run while it is stored.
             // A thread holds one row; to store whole 128-byte row segments the warp passes each 32 x 32 block
@@ -651,13 +709,13 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
             float4* stg = reinterpret_cast<float4*>(smem_raw + (bars + 256u - smem_u32(smem_raw))) + (warp - 2) * 256;
 #pragma unroll
             for (int g = 0; g < ACC_REGS / 32; ++g) {
+                if (ks > 1 && (col0 + 32 * g) / (BN / ks) != kpart) continue;  // another CTA of the cluster stores this block
                 __syncwarp();
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
                     stg[lane * 8 + (k ^ (lane & 7))] =
                         make_float4(acc[32 * g + 4 * k], acc[32 * g + 4 * k + 1], acc[32 * g + 4 * k + 2], acc[32 * g + 4 * k + 3]);
                 __syncwarp();
-                if (ks > 1 && (col0 + 32 * g) / (BN / ks) != kpart) continue;  // another CTA of the cluster stores this block
                 store_block(args, stg, br, m0 + q * 32, n0 + col0 + 32 * g, CPW - 32 * g, lane);
             }
         }
