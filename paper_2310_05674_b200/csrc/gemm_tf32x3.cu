@@ -265,6 +265,10 @@ struct TcArgs {
     int branches;          // 1 or 2; a work item is (branch, tile)
     int ksplit;            // single-CTA tiles only: CTAs of a cluster that share one tile's contraction (1, 2 or 4)
     float4* ws;            // ksplit > 1: partial tiles, [item][ksplit][128 x BN floats]
+    // Pair tiles only: when the tiles do not fill the last round, every unit first takes `full_rounds` whole
+    // tiles, then the `tail_tiles` remaining ones are each shared by two units (half of the k-blocks each).
+    int full_rounds, tail_tiles;
+    int* flags;            // arrival counters of the shared tail tiles [tail tile][2 halves][2 CTAs], zero between launches
     uint32_t tx_bytes;     // bytes the four copies of one k-block deliver
     int32_t* status;
 };
@@ -422,6 +426,27 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     const int kb_per_part = (args.num_kb + ks - 1) / ks;
     const int kb_begin = kpart * kb_per_part;
     const int num_kb = min(kb_per_part, args.num_kb - kb_begin);
+    // The step-th piece of work of this unit: a tile and a range of its k-blocks.  tpart >= 0: a tail tile
+    // shared with another pair, of which this is half `tpart`.
+    auto next_work = [&](int step, int& item, int& kb0, int& nkb, int& tpart) -> bool {
+        tpart = -1;
+        if (PAIR && args.tail_tiles > 0) {
+            if (step < args.full_rounds) { item = unit + step * n_units; kb0 = 0; nkb = args.num_kb; return true; }
+            if (step == args.full_rounds && unit < 2 * args.tail_tiles) {
+                item = args.full_rounds * n_units + (unit >> 1);
+                tpart = unit & 1;
+                const int half = (args.num_kb + 1) / 2;
+                kb0 = tpart * half;
+                nkb = tpart ? args.num_kb - half : half;
+                return true;
+            }
+            return false;
+        }
+        item = unit + step * n_units;
+        kb0 = kb_begin;
+        nkb = num_kb;
+        return item < n_items;
+    };
     // Work item -> branch and tile origin.  Tile order inside a branch: items that run together cover all
     // M-tiles of a group of `group_n` N-tiles, so one wave re-uses a bounded set of W tiles and every A tile
     // from L2 instead of sweeping all of W.
@@ -454,7 +479,8 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
             mbar_init(acc_empty_bar(b), EPI * (PAIR ? 2 : 1));  // one arrival per epilogue warp (of both CTAs of a pair)
         }
         mbar_init(part_bar, EPI * (ks > 1 ? ks - 1 : 1));       // one arrival per epilogue warp of every other CTA
-        *abort_flag = 0;
+        abort_flag[0] = 0;
+        abort_flag[1] = 0;  // epilogue warps that have finished the exchange of a shared tail tile
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -482,15 +508,17 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
             int s = 0;
             uint32_t empty_parity = 1;  // parity of the phase that frees stage s for its next round
             bool ok = true;
-            for (int item = unit; item < n_items && ok; item += n_units) {
+            for (int step = 0; ok; ++step) {
+                int item, kb0, nkb, tpart;
+                if (!next_work(step, item, kb0, nkb, tpart)) break;
                 int br, m0, n0;
                 locate(item, br, m0, n0);
                 const int nw0 = n0 + (int)rank * WROWS;  // first W row this CTA stages
                 const int za = args.shared_a ? 0 : br;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = 0; kb < nkb; ++kb) {
                     if (issued >= STAGES && !mbar_wait(empty_bar(s), empty_parity, abort_flag)) { raise_timeout(); ok = false; break; }
                     const uint32_t st = base + s * STAGE;
-                    const int kx = (kb_begin + kb) * BKF;
+                    const int kx = (kb0 + kb) * BKF;
                     if (PAIR) {
                         // both CTAs' copies complete on the leader's barrier, which the leader arms for all of them
                         const uint32_t lbar = full_bar(s) & kPeerBitMask;
@@ -522,9 +550,11 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
             bool ok = true;
             int s = 0, chunk = 0;  // chunk counts over all of this CTA's tiles: accumulator = chunk & 1
             uint32_t full_parity = 0;
-            for (int item = unit; item < n_items && ok; item += n_units) {
+            for (int step = 0; ok; ++step) {
+                int item, kb0, nkb, tpart;
+                if (!next_work(step, item, kb0, nkb, tpart)) break;
                 int in_chunk = 0;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = 0; kb < nkb; ++kb) {
                     const int buf = chunk & 1;
                     const bool chunk_first = in_chunk == 0;
                     if (chunk_first && chunk >= 2) {
@@ -556,7 +586,7 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                     }
                     // frees the stage (in both CTAs of a pair) once these products have read it
                     if (PAIR) umma_commit_pair(empty_bar(s)); else umma_commit(empty_bar(s));
-                    if (in_chunk == kChunkKb - 1 || kb == num_kb - 1) {
+                    if (in_chunk == kChunkKb - 1 || kb == nkb - 1) {
                         if (PAIR) umma_commit_pair(acc_full_bar(buf)); else umma_commit(acc_full_bar(buf));
                         in_chunk = 0;
                         ++chunk;
@@ -572,12 +602,18 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         const int q = warp & 3;            // a warp may only touch TMEM lanes [32 q, 32 q + 32)
         const int col0 = ((warp - 2) >> 2) * CPW;  // with eight epilogue warps, two share a lane quarter and split the columns
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)col0;
-        const int n_chunks = (num_kb + kChunkKb - 1) / kChunkKb;
-        const int my_items = unit < n_items ? (n_items - unit + n_units - 1) / n_units : 0;
-        const int total_chunks = my_items * n_chunks;
+        int total_chunks = 0;
+        for (int step = 0;; ++step) {
+            int item, kb0, nkb, tpart;
+            if (!next_work(step, item, kb0, nkb, tpart)) break;
+            total_chunks += (nkb + kChunkKb - 1) / kChunkKb;
+        }
         int chunk = 0;  // counts over all of this CTA's tiles, like the issuer's
         bool ok = true;
-        for (int item = unit; item < n_items && ok; item += n_units) {
+        for (int step = 0; ok; ++step) {
+            int item, kb0, nkb, tpart;
+            if (!next_work(step, item, kb0, nkb, tpart)) break;
+            const int n_chunks = (nkb + kChunkKb - 1) / kChunkKb;
             int br, m0, n0;
             locate(item, br, m0, n0);
             float acc[ACC_REGS];
@@ -703,6 +739,47 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                 }
                 }
             }
+            if (PAIR && tpart >= 0) {
+                // A tail tile shared with another pair (a separate cluster): each CTA leaves the column half it
+                // does not own in the workspace, counts its arrival in global memory, waits (bounded) for the
+                // CTA of the same pair rank in the other pair, and adds that CTA's partial sums to its own half.
+                // Every pair of the launch is resident and this is its last tile, so the wait cannot cycle.
+                const int t = item - args.full_rounds * n_units;
+                const int wi = warp - 2;
+                const int other = tpart ^ 1;
+                float4* slabs = args.ws + ((size_t)t * 4 + rank) * (BM * BN / 4) + (wi * (CPW / 4)) * 32 + lane;
+                float4* mine = slabs + (size_t)tpart * 2 * (BM * BN / 4);
+                const bool sender = (col0 / (BN / 2)) != tpart;   // (CPW = BN / 2: a warp's columns lie in one half)
+                if (sender) {
+#pragma unroll
+                    for (int k = 0; k < CPW / 4; ++k)
+                        __stcg(mine + k * 32, make_float4(acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]));
+                }
+                __threadfence();
+                __syncwarp();
+                int* my_flag = args.flags + ((t * 2 + tpart) * 2 + (int)rank);
+                if (lane == 0) {
+                    atomicAdd(args.flags + ((t * 2 + other) * 2 + (int)rank), 1);
+                    const long long t0 = clock64();
+                    while (*reinterpret_cast<volatile int*>(my_flag) < EPI) {
+                        if (*abort_flag) { ok = false; break; }
+                        if (clock64() - t0 > 2 * kWaitCycles) { raise_timeout(); ok = false; break; }
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                __threadfence();
+                if (!sender) {
+                    const float4* theirs = slabs + (size_t)other * 2 * (BM * BN / 4);
+#pragma unroll
+                    for (int k = 0; k < CPW / 4; ++k) {
+                        const float4 v = __ldcg(theirs + k * 32);
+                        acc[4 * k] += v.x; acc[4 * k + 1] += v.y; acc[4 * k + 2] += v.z; acc[4 * k + 3] += v.w;
+                    }
+                }
+                // the last of this CTA's epilogue warps to get here puts the counter back to zero
+                if (lane == 0 && atomicAdd(const_cast<uint32_t*>(abort_flag + 1), 1u) == (uint32_t)(EPI - 1)) *my_flag = 0;
+            }
             // The tile's sum is in registers; the products of the next tile already run while it is stored.
             // A thread holds one row; to store whole 128-byte row segments the warp passes each 32 x 32 block
             // through shared memory (16-byte chunks XOR-swizzled by row: no bank conflicts either way).
@@ -710,6 +787,7 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
 #pragma unroll
             for (int g = 0; g < ACC_REGS / 32; ++g) {
                 if (ks > 1 && (col0 + 32 * g) / (BN / ks) != kpart) continue;  // another CTA of the cluster stores this block
+                if (PAIR && tpart >= 0 && (col0 + 32 * g) / (BN / 2) != tpart) continue;  // the other pair stores it
                 __syncwarp();
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
@@ -846,7 +924,8 @@ bool make_map(CUtensorMap* map, const float* base, int ld, int64_t rows, int sla
 
 // Launches the persistent kernel on min(work items, co-resident CTAs or CTA pairs) units.
 template <int BN, bool PAIR, int EPI>
-cudaError_t launch_tc(const CUtensorMap maps[4], const TcArgs& a, int items, int sm_count, cudaStream_t st) {
+cudaError_t launch_tc(const CUtensorMap maps[4], const TcArgs& a, int items, int sm_count, cudaStream_t st,
+                      size_t ws_floats = 0, int tail_flags = 0) {
     const int ks = PAIR ? 1 : a.ksplit;
     constexpr int kSmem = smem_bytes(PAIR ? BN / 2 : BN);
     static int max_units = 0;  // one CTA per SM (shared memory); pairs: what the cluster scheduler can co-schedule
@@ -879,8 +958,22 @@ cudaError_t launch_tc(const CUtensorMap maps[4], const TcArgs& a, int items, int
         return launch_clustered(ks, gemm_tf32x3_kernel<BN, PAIR, EPI>, dim3(items * ks), dim3(threads_for(EPI)),
                                 (size_t)kSmem, st, maps[0], maps[1], maps[2], maps[3], a);
     const int units = items < max_units ? items : max_units;
+    TcArgs b = a;
+    b.full_rounds = 0;
+    b.tail_tiles = 0;
+    if (PAIR && items > max_units) {
+        // tiles that do not fill the last round are each shared by two pairs when that takes no more pairs
+        // than there are (and the contraction is long enough to be worth an exchange)
+        const int rounds = items / max_units, tail = items % max_units;
+        static const bool off = []() { const char* e = std::getenv("SAMA_TC_TAIL"); return e && e[0] == '0'; }();
+        if (!off && tail > 0 && 2 * tail <= max_units && a.num_kb >= 16 && a.flags && tail * 4 <= tail_flags &&
+            (size_t)tail * 4 * BM * BN <= ws_floats) {
+            b.full_rounds = rounds;
+            b.tail_tiles = tail;
+        }
+    }
     return launch_clustered(PAIR ? 2 : 1, gemm_tf32x3_kernel<BN, PAIR, EPI>, dim3(units * (PAIR ? 2 : 1)),
-                            dim3(threads_for(EPI)), (size_t)kSmem, st, maps[0], maps[1], maps[2], maps[3], a);
+                            dim3(threads_for(EPI)), (size_t)kSmem, st, maps[0], maps[1], maps[2], maps[3], b);
 }
 
 inline int round_up32(int x) { return (x + 31) & ~31; }
@@ -1005,6 +1098,9 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     a.branches = nbr;
     a.ksplit = pair ? 1 : ksplit;
     a.ws = reinterpret_cast<float4*>(ctx->tc_ws);
+    a.flags = ctx->tc_flags;
+    a.full_rounds = 0;
+    a.tail_tiles = 0;
     // about one wave of CTAs per group: group_n N-tiles x all M-tiles
     a.group_n = ctx->sm_count / a.tiles_m;
     if (a.group_n < 1) a.group_n = 1;
@@ -1017,7 +1113,7 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     // its small kernels (the direct gradient, see run_meta_grad_tc).
     PdlScope pdl(pdl_enabled() ? 1 : 0);
     // eight epilogue warps (two per lane quarter, each taking half of the columns) except on the 16-wide tile
-    if (pair) return launch_tc<256, true, 8>(maps, a, items, sms, st);
+    if (pair) return launch_tc<256, true, 8>(maps, a, items, sms, st, ctx->tc_ws_floats, ctx->tc_flags ? kTcFlags : 0);
     if (bn == 16) return launch_tc<16, false, 4>(maps, a, items, sms, st);
     if (bn == 64) return launch_tc<64, false, 8>(maps, a, items, sms, st);
     return launch_tc<128, false, 8>(maps, a, items, sms, st);

@@ -391,8 +391,10 @@ int sama_create(sama_ctx** out, int device, int64_t max_n, int32_t max_batch, co
         ctx->a_split_half = 2 * (size_t)max_batch * amax;
         ok = ok && cudaMalloc(&ctx->x_split, sizeof(float) * 2 * ctx->x_split_half) == cudaSuccess &&
              cudaMalloc(&ctx->w_split, sizeof(float) * 2 * ctx->w_split_half) == cudaSuccess;
-        ctx->tc_ws_floats = (size_t)ctx->sm_count * 128 * 128;
-        ok = ok && cudaMalloc(&ctx->tc_ws, sizeof(float) * ctx->tc_ws_floats) == cudaSuccess;
+        ctx->tc_ws_floats = (size_t)ctx->sm_count * 128 * 256;
+        ok = ok && cudaMalloc(&ctx->tc_ws, sizeof(float) * ctx->tc_ws_floats) == cudaSuccess &&
+             cudaMalloc(&ctx->tc_flags, sizeof(int) * kTcFlags) == cudaSuccess &&
+             cudaMemset(ctx->tc_flags, 0, sizeof(int) * kTcFlags) == cudaSuccess;
         ctx->mg_ws_floats = meta_grad_workspace_floats(mlp, max_batch);
         ok = ok && cudaMalloc(&ctx->mg_ws, sizeof(float) * ctx->mg_ws_floats) == cudaSuccess;
         ctx->mg_tc_floats = meta_grad_tc_floats(mlp, max_batch);
@@ -423,6 +425,7 @@ int sama_destroy(sama_ctx* ctx) {
     cudaFree(ctx->a_split[0]);
     cudaFree(ctx->a_split[1]);
     cudaFree(ctx->tc_ws);
+    cudaFree(ctx->tc_flags);
     cudaFree(ctx->mg_ws);
     cudaFree(ctx->mg_tc);
     cudaFree(ctx->stage);

@@ -11,6 +11,7 @@ namespace sama {
 
 constexpr int kMaxLayers = 16;
 constexpr int kMaxPartials = 4096;  // upper bound on the grid of the reduction kernels
+constexpr int kTcFlags = 1024;      // arrival counters of the tensor-core kernel's shared tail tiles
 
 // Device scalars owned by a context.
 struct DeviceScalars {
@@ -85,7 +86,8 @@ struct sama_ctx {
     float* w_split;                // device [hi, lo][2 branches][slab]: every layer's W, rows padded to 32
     float* a_split[2];             // device, ping-pong: [2][2][max_batch][round32(max hidden)]
     size_t x_split_half, w_split_half, a_split_half;  // floats per hi (or lo) part; 0 = path unavailable
-    float* tc_ws;                  // device: partial tiles of the tensor-core path's K-split (one 128 x 128 tile per SM)
+    float* tc_ws;                  // device: partial tiles of the tensor-core path's K-split (one 128 x 256 tile per SM)
+    int* tc_flags;                 // device [kTcFlags], zero between launches
     size_t tc_ws_floats;
     float* mg_ws;                  // device: workspace of the direct gradient (activations, dz, losses)
     size_t mg_ws_floats;

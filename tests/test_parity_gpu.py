@@ -301,6 +301,21 @@ def test_several_tiles_per_cta(monkeypatch, pairs):
     assert np.array_equal(a["metagrad"], b["metagrad"]) and np.array_equal(a["loss_plus"], b["loss_plus"])
 
 
+def test_shared_tail_tiles_of_the_pair_kernel():
+    """100 pair tiles on 74 resident CTA pairs: after one full round the 26 remaining tiles are each
+    shared by two pairs (half of the 16 k-blocks each), which exchange partial sums through the
+    workspace with arrival counters in global memory.  Same parity bar, bitwise repeatable, counters
+    back at zero (the second and third call reuse them)."""
+    cfg, w = W.custom_mlp((512, 2560, 40), 1280, seed=9)
+    check_step(cfg, w, B.Adam(), 1.0, gemm_mode=2)
+    with Ctx(cfg.n_params, cfg.batch, cfg.dims, 2) as ctx:
+        a = run_step(ctx, cfg, w, B.Adam(), 1.0)
+        b = run_step(ctx, cfg, w, B.Adam(), 1.0)
+        c = run_step(ctx, cfg, w, B.Adam(), 1.0)
+    assert a["status"] == 0 and c["status"] == 0
+    assert np.array_equal(a["metagrad"], b["metagrad"]) and np.array_equal(a["loss_plus"], c["loss_plus"])
+
+
 def test_step_host_matches_step():
     cfg = W.CONFIGS["tiny"]
     w = W.mlp_workload(cfg, 0)
