@@ -59,7 +59,8 @@ typedef enum sama_status {
 enum {
     SAMA_DEV_DEGENERATE_NORM = 1, /* ||p|| was 0 or not finite: eps_fd = 0, theta+- = theta, metagrad = 0 */
     SAMA_DEV_BAD_LABEL = 2,       /* a label outside [0, d_L): that sample's metagrad is 0 */
-    SAMA_DEV_TIMEOUT = 4          /* a bounded wait inside a kernel expired; outputs of that call are invalid */
+    SAMA_DEV_TIMEOUT = 4          /* a bounded wait inside a kernel expired; outputs of that call are invalid, and the
+                                     context's arrival counters may be left non-zero: destroy and recreate it */
 };
 
 /* Base optimiser state that the adaptation differentiates (Appendix C).
