@@ -20,6 +20,7 @@ pretrained weights, none of which is used.
 """
 from __future__ import annotations
 
+import os
 from concurrent.futures import ThreadPoolExecutor
 from dataclasses import dataclass, field
 from typing import Dict, List, Optional, Sequence, Tuple
@@ -44,6 +45,12 @@ STREAM_FLIP = 8
 STREAM_FLIP_TO = 9
 STREAM_LAMBDA = 10
 STREAM_MEANS = 11
+STREAM_REG_X = 12
+STREAM_REG_XV = 13
+STREAM_REG_W = 14
+STREAM_REG_NOISE = 15
+STREAM_REG_NOISE_V = 16
+STREAM_REG_LAMBDA = 17
 
 
 def _mix64(z: np.ndarray) -> np.ndarray:
@@ -91,7 +98,7 @@ def _chunked(fn, seed: int, stream: int, n: int, offset: int, dtype) -> np.ndarr
     if len(spans) == 1:
         work(spans[0])
     else:
-        with ThreadPoolExecutor(max_workers=8) as ex:
+        with ThreadPoolExecutor(max_workers=min(32, os.cpu_count() or 8)) as ex:
             list(ex.map(work, spans))
     return out
 
@@ -253,3 +260,38 @@ def custom_mlp(dims: Sequence[int], batch: int, seed: int, noise_rate: float = 0
     """A workload of arbitrary (e.g. ragged) shape with the same recipe."""
     cfg = MLPConfig(name, tuple(int(d) for d in dims), int(batch), noise_rate)
     return cfg, mlp_workload(cfg, seed)
+
+
+# --------------------------------------------------------------------------
+# Biased regression (the setting of the paper's Appendix E; its sizes are not stated there)
+# --------------------------------------------------------------------------
+
+@dataclass
+class BiasRegConfig:
+    name: str
+    d: int          # features = dim(w) = dim(lambda)
+    n: int          # base (training) samples
+    n_val: int      # meta (validation) samples
+    beta: float = 0.1
+    noise: float = 0.1
+    meta_updates: int = 100
+
+
+BIASREG: Dict[str, BiasRegConfig] = {
+    "biasreg256": BiasRegConfig("biasreg256", 256, 512, 512),
+    "biasreg4096": BiasRegConfig("biasreg4096", 4096, 8192, 8192),
+}
+
+
+def biased_regression(cfg: BiasRegConfig, seed: int = 0) -> Dict[str, np.ndarray]:
+    """X, X' ~ N(0, 1) entrywise scaled by 1/sqrt(d); y = X w_true + noise z, y' = X' w_true + noise z';
+    w_true ~ N(0, 1); lambda_0 ~ N(0, 1).  All fp32."""
+    d, n, nv = cfg.d, cfg.n, cfg.n_val
+    sc = 1.0 / np.sqrt(d)
+    X = (sc * normal(seed, STREAM_REG_X, n * d)).astype(np.float32).reshape(n, d)
+    Xv = (sc * normal(seed, STREAM_REG_XV, nv * d)).astype(np.float32).reshape(nv, d)
+    w_true = normal(seed, STREAM_REG_W, d)
+    y = (X.astype(np.float64) @ w_true + cfg.noise * normal(seed, STREAM_REG_NOISE, n)).astype(np.float32)
+    yv = (Xv.astype(np.float64) @ w_true + cfg.noise * normal(seed, STREAM_REG_NOISE_V, nv)).astype(np.float32)
+    lam0 = normal(seed, STREAM_REG_LAMBDA, d).astype(np.float32)
+    return {"X": X, "y": y, "Xv": Xv, "yv": yv, "lam0": lam0, "w_true": w_true.astype(np.float32)}
