@@ -15,6 +15,8 @@ MUTATIONS = {
     "eps_term_always_dropped": ("if (!h->drop_eps_term) num +=", "if (false) num +="),
     "missing_sqrt_c2_in_denominator": ("num / (rc2 * r * D * D)", "num / (r * D * D)"),
     "no_bias_correction_in_D": ("const double D = r / rc2 + eps;", "const double D = r + eps;"),
+    "dropped_eps_form_keeps_exact_value_at_zero_state": ("J = h->drop_eps_term ? 0.0 : (h->lr / c1) * (1.0 - b1) / eps;",
+                                                         "J = (h->lr / c1) * (1.0 - b1) / eps;"),
     "missing_c1": ("J = (h->lr / c1) * num", "J = (h->lr) * num"),
     "second_moment_uses_beta1": ("b2 * sk + (1.0 - b2) * g * g", "b1 * sk + (1.0 - b1) * g * g"),
     "gbase_ignored": ("const double g = g_base ? (double)g_base[k] : mk;", "const double g = mk;"),

@@ -108,6 +108,40 @@ def test_zero_state_limit():
     assert jac(0.0, 0.0, 0.0, adam) == pytest.approx(float(d), rel=1e-4)
 
 
+def test_zero_state_value_of_the_printed_approximation():
+    """drop_eps_term at s = 0 and g = 0 (r = 0), where the printed approximate form (Appendix C, last
+    line) is 0/0.  The checker returns 0 there.  That is what the form itself fixes: along g = 0 it is
+    lr (1-b1) r / (c1 sqrt(c2) D^2) with r^2 = b2 s, which goes to 0 with s; along s = 0 it tends to
+    -+ lr b1 sqrt(1-b2) m / (c1 sqrt(c2) eps^2) for g -> 0+-, two one-sided limits whose mean is 0 (the same
+    symmetric-derivative convention that gives the exact form its value (lr/c1)(1-b1)/eps at this point).
+    Both statements are evaluated from the formula typed out here, and against the checker just off the point."""
+    lr, b1, b2, eps, step = 1e-3, 0.9, 0.999, 1e-8, 10
+    c1, c2 = 1 - b1 ** step, 1 - b2 ** step
+    adam = oracle.Adam(lr, b1, b2, eps, step, drop_eps_term=True)
+    for m in (0.0, 3e-4, -2e-3):
+        assert jac(m, 0.0, 0.0, adam) == 0.0
+        # along g = 0, once r is below eps: monotone to 0 with s, and equal to the typed-out expression
+        prev = None
+        for s in (1e-18, 1e-22, 1e-26, 1e-32, 1e-37):
+            sd = float(np.float32(s))
+            r = np.sqrt(b2 * sd)
+            D = r / np.sqrt(c2) + eps
+            expect = (lr / c1) * (1 - b1) * b2 * sd / (np.sqrt(c2) * r * D * D)
+            J = jac(m, s, 0.0, adam)
+            assert J == pytest.approx(expect, rel=1e-12)
+            assert prev is None or abs(J) < abs(prev)
+            prev = J
+        assert abs(prev) < 1e-8 * (lr / c1) * (1 - b1) / eps
+        # along s = 0: odd in g, with the one-sided limits typed out
+        for g in (1e-20, 1e-24):
+            Jp, Jm = jac(m, 0.0, g, adam), jac(m, 0.0, -g, adam)
+            md = float(np.float32(m))
+            lim = -(lr / c1) * b1 * np.sqrt(1 - b2) * md / (np.sqrt(c2) * eps ** 2)
+            assert Jp == pytest.approx(lim, rel=1e-6, abs=1e-12)
+            assert Jm == pytest.approx(-lim, rel=1e-6, abs=1e-12)
+            assert Jp + Jm == pytest.approx(0.0, abs=1e-6 * max(abs(lim), 1e-12))
+
+
 def test_identity_mode_is_bit_exact_and_sgd_reduction():
     w = W.adam_state(1000, 3)
     p = oracle.adapt(w["m"], w["s"], w["g_base"], w["g_meta"], oracle.Adam(identity=True))
