@@ -68,6 +68,10 @@ def _bind(lib):
     lib.sama_oracle_fd.restype = None
     lib.sama_oracle_meta_grad.argtypes = [C.c_int32, ip, fp, fp, ip, C.c_int32, dp]
     lib.sama_oracle_meta_grad.restype = C.c_double
+    lib.sama_oracle_reweight_grad.argtypes = [C.c_int32, dp, C.c_int32, fp, C.c_int32, dp, dp]
+    lib.sama_oracle_reweight_grad.restype = None
+    lib.sama_oracle_fd_reweight.argtypes = [C.c_int32, dp, dp, C.c_int32, fp, C.c_double, C.c_int32, dp]
+    lib.sama_oracle_fd_reweight.restype = None
     lib.sama_oracle_step.argtypes = [C.c_int32, ip, C.c_int64, fp, fp, fp, fp, fp, ap, C.c_double,
                                      fp, ip, fp, C.c_int32, C.c_int32, dp, dp, dp, dp, dp, dp, dp]
     lib.sama_oracle_step.restype = C.c_int
@@ -166,6 +170,30 @@ def fd(loss_plus, loss_minus, lam, eps_fd: float, B_norm: int) -> np.ndarray:
     out = np.empty(lp.size, dtype=np.float64)
     _load().sama_oracle_fd(lp.size, _p(lp, C.c_double), _p(lm, C.c_double), _p(lam, C.c_float),
                            float(eps_fd), int(B_norm), _p(out, C.c_double))
+    return out
+
+
+def reweight_grad(loss, lambda_r, B_norm: Optional[int] = None):
+    """dL_base/dlambda_r at fixed theta for the shared reweighting network of Sec. 4.1
+    (lambda_r = v1[H], c1[H], v2[H], c2); returns (gradient [3H + 1], per-sample weights)."""
+    loss, lambda_r = _f64(loss), _f32(lambda_r)
+    H = (lambda_r.size - 1) // 3
+    assert lambda_r.size == 3 * H + 1
+    g, wts = np.empty(3 * H + 1, dtype=np.float64), np.empty(loss.size, dtype=np.float64)
+    _load().sama_oracle_reweight_grad(loss.size, _p(loss, C.c_double), H, _p(lambda_r, C.c_float),
+                                      int(loss.size if B_norm is None else B_norm), _p(g, C.c_double),
+                                      _p(wts, C.c_double))
+    return g, wts
+
+
+def fd_reweight(loss_plus, loss_minus, lambda_r, eps_fd: float, B_norm: Optional[int] = None) -> np.ndarray:
+    """Eq. 5 with the shared reweighting network: central difference of dL_base/dlambda_r between theta+ and theta-."""
+    lp, lm, lambda_r = _f64(loss_plus), _f64(loss_minus), _f32(lambda_r)
+    H = (lambda_r.size - 1) // 3
+    assert lambda_r.size == 3 * H + 1
+    out = np.empty(3 * H + 1, dtype=np.float64)
+    _load().sama_oracle_fd_reweight(lp.size, _p(lp, C.c_double), _p(lm, C.c_double), H, _p(lambda_r, C.c_float),
+                                    float(eps_fd), int(lp.size if B_norm is None else B_norm), _p(out, C.c_double))
     return out
 
 

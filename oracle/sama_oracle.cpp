@@ -36,6 +36,11 @@
 // mixed second derivative on a linear-softmax model with O(alpha^2) error
 // decay; brute-force nested differences on tiny MLPs; forward pass against a
 // library matmul; antisymmetry, scaling and permutation invariants.
+// The shared reweighting network of Sec. 4.1 (sama_oracle_reweight_grad, sama_oracle_fd_reweight) is pinned in
+// tests/test_oracle_reweight_pins.py: extended-precision differences of the base objective in lambda_r,
+// hand-computed special cases, nested differences on tiny MLPs.  Reading: the paper says "2-layer MLP" and
+// gives neither width nor activations; ReLU hidden units and a sigmoid output are taken (as in the
+// reweighting network the paper cites), the width is an argument.
 // No function here is "parity unpinned".
 
 #include <cmath>
@@ -227,6 +232,57 @@ void sama_oracle_fd(int32_t count, const double* loss_plus, const double* loss_m
         const double sg = 1.0 / (1.0 + std::exp(-(double)lambda[i]));
         metagrad_out[i] = -sg * (1.0 - sg) * (loss_plus[i] - loss_minus[i]) / (2.0 * eps_fd * (double)B_norm);
     }
+}
+
+// Shared reweighting network -- the meta learner of Sec. 4.1, w(l; lambda_r): a 2-layer MLP on the
+// scalar per-sample loss l with H hidden units and a sigmoid output,
+//   a_j = v1_j l + c1_j,  h_j = max(0, a_j),  z = sum_j v2_j h_j + c2,  w = sigmoid(z),
+// lambda_r = (v1[H], c1[H], v2[H], c2) in that order (3H + 1 numbers).  The base objective is
+//   L_base(theta, lambda_r) = (1/B) sum_i w(l_i(theta); lambda_r) l_i(theta),
+// so at fixed theta
+//   dL_base/dlambda_r = (1/B) sum_i l_i w_i (1 - w_i) dz_i/dlambda_r,
+//   dz/dc2 = 1,  dz/dv2_j = h_j,  dz/dc1_j = v2_j [a_j > 0],  dz/dv1_j = v2_j [a_j > 0] l.
+// grad_out has 3H + 1 entries; weights_out (count entries, may be null) receives w_i.
+void sama_oracle_reweight_grad(int32_t count, const double* loss, int32_t H, const float* lambda_r,
+                               int32_t B_norm, double* grad_out, double* weights_out) {
+    const float* v1 = lambda_r;
+    const float* c1 = lambda_r + H;
+    const float* v2 = lambda_r + 2 * (int64_t)H;
+    const double c2 = (double)lambda_r[3 * (int64_t)H];
+    for (int32_t k = 0; k < 3 * H + 1; ++k) grad_out[k] = 0.0;
+    for (int32_t i = 0; i < count; ++i) {
+        const double l = loss[i];
+        double z = c2;
+        for (int32_t j = 0; j < H; ++j) {
+            const double a = (double)v1[j] * l + (double)c1[j];
+            if (a > 0.0) z += (double)v2[j] * a;
+        }
+        const double w = 1.0 / (1.0 + std::exp(-z));
+        if (weights_out) weights_out[i] = w;
+        const double f = l * w * (1.0 - w) / (double)B_norm;
+        for (int32_t j = 0; j < H; ++j) {
+            const double a = (double)v1[j] * l + (double)c1[j];
+            if (a > 0.0) {
+                grad_out[j] += f * (double)v2[j] * l;          // v1_j
+                grad_out[H + j] += f * (double)v2[j];          // c1_j
+                grad_out[2 * (int64_t)H + j] += f * a;          // v2_j
+            }
+        }
+        grad_out[3 * (int64_t)H] += f;                          // c2
+    }
+}
+
+// Eq. 5 with the shared reweighting network as the meta learner:
+//   metagrad = -[ dL_base(theta+)/dlambda_r - dL_base(theta-)/dlambda_r ] / (2 eps_fd),
+// from the per-sample losses at theta+ and theta- (S4).  3H + 1 entries; zero when eps_fd is not positive.
+void sama_oracle_fd_reweight(int32_t count, const double* loss_plus, const double* loss_minus, int32_t H,
+                             const float* lambda_r, double eps_fd, int32_t B_norm, double* metagrad_out) {
+    const int32_t dim = 3 * H + 1;
+    std::vector<double> gp(dim), gm(dim);
+    sama_oracle_reweight_grad(count, loss_plus, H, lambda_r, B_norm, gp.data(), nullptr);
+    sama_oracle_reweight_grad(count, loss_minus, H, lambda_r, B_norm, gm.data(), nullptr);
+    for (int32_t k = 0; k < dim; ++k)
+        metagrad_out[k] = eps_fd > 0.0 ? -(gp[k] - gm[k]) / (2.0 * eps_fd) : 0.0;
 }
 
 // S1..S5 chained (the workflow of Fig. 2 with lambda = per-sample weights).

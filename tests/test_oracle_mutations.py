@@ -8,6 +8,7 @@ import pytest
 
 import oracle
 import test_oracle_pins as pins
+import test_oracle_reweight_pins as reweight_pins
 
 MUTATIONS = {
     "garbled_mg_coefficients": ("b1 * (1.0 - b2) * mk * g", "(1.0 - b1) * b2 * mk * g"),
@@ -35,10 +36,19 @@ MUTATIONS = {
     "meta_grad_no_onehot": ("(c == y[i] ? 1.0 : 0.0)", "0.0"),
     "meta_grad_transposed_backprop": ("dh[k] += (double)theta[woff[l] + (int64_t)j * din + k] * dz[j];",
                                       "dh[k] += (double)theta[woff[l] + ((int64_t)k * dout + j) % ((int64_t)din * dout)] * dz[j];"),
+    "reweight_sigmoid_derivative_dropped": ("const double f = l * w * (1.0 - w) / (double)B_norm;",
+                                            "const double f = l * w / (double)B_norm;"),
+    "reweight_loss_factor_dropped": ("const double f = l * w * (1.0 - w) / (double)B_norm;",
+                                     "const double f = w * (1.0 - w) / (double)B_norm;"),
+    "reweight_relu_mask_dropped": ("            if (a > 0.0) {\n                grad_out[j] += f", "            if (true) {\n                grad_out[j] += f"),
+    "reweight_v1_gradient_without_input": ("grad_out[j] += f * (double)v2[j] * l;", "grad_out[j] += f * (double)v2[j];"),
+    "reweight_v2_gradient_uses_weight": ("grad_out[2 * (int64_t)H + j] += f * a;", "grad_out[2 * (int64_t)H + j] += f * (double)v2[j];"),
+    "reweight_fd_sign": ("eps_fd > 0.0 ? -(gp[k] - gm[k])", "eps_fd > 0.0 ? (gp[k] - gm[k])"),
+    "reweight_fd_one_sided_scale": ("(gp[k] - gm[k]) / (2.0 * eps_fd)", "(gp[k] - gm[k]) / (eps_fd)"),
     "no_batch_mean": ("(2.0 * eps_fd * (double)B_norm)", "(2.0 * eps_fd)"),
 }
 
-PINS = [getattr(pins, n) for n in dir(pins) if n.startswith("test_")]
+PINS = [getattr(mod, n) for mod in (pins, reweight_pins) for n in dir(mod) if n.startswith("test_")]
 
 
 def _run_all_pins():
