@@ -129,6 +129,9 @@ int sama_adapt(sama_ctx* ctx, int64_t n, const float* m, const float* s, const f
  *     stream at the start of each call, so calls issued one after another on
  *     one stream are safe; calls that can overlap on the GPU (different
  *     streams, no ordering) race on it and give wrong sums.
+ *   - the resolved address is remembered for the life of the process; after a
+ *     cudaDeviceReset on that device it is stale, and this entry point must
+ *     not be called again in that process.
  * Calls cudaGetDevice, cudaGetSymbolAddress / cudaDeviceGetAttribute (first
  * call only), cudaMemsetAsync and one kernel launch; never cudaMalloc or
  * cudaFree. */
@@ -166,7 +169,11 @@ int sama_fd_metagrad(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_pl
  * sama_adapt -> sama_perturb -> sama_fd_metagrad on one stream, no host
  * synchronisation in between.  n must equal the parameter count of mlp.
  * Outputs: p_out [n] (may alias g_meta), theta_plus [n], theta_minus [n] (may
- * alias theta), metagrad_out [B]; loss_*_out optional. */
+ * alias theta), metagrad_out [B]; loss_*_out optional.  theta_plus and / or
+ * theta_minus may be NULL when the caller has no use for them: the tensor-core
+ * forward reads its own operand copies, so a NULL output is then never written
+ * to memory at all (4 B/element less traffic each); on the fp32 FMA path the
+ * context keeps it in scratch allocated on first use (cudaMalloc; synchronises). */
 int sama_step(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* theta, const float* m,
               const float* s, const float* g_base, const float* g_meta, const sama_adam_t* adam, float alpha,
               const float* X, const int32_t* y, const float* lambda, int32_t B,
@@ -182,6 +189,60 @@ int sama_step(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* thet
  * with an mlp whose layer widths are not smaller, B <= max_batch.  Results are reproducible bit for bit. */
 int sama_meta_grad(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta, const float* X_meta,
                    const int32_t* y_meta, int32_t B, float* g_meta_out, float* loss_out, void* stream);
+
+/* Eq. 5 when the meta learner is a shared reweighting network w(l; lambda_r) (Sec. 4.1) instead of
+ * per-sample logits:  L_base = (1/B) sum_i w(l_i(theta); lambda_r) l_i(theta),  w a 2-layer MLP on the
+ * scalar loss,  a_j = v1_j l + c1_j,  z = sum_j v2_j max(0, a_j) + c2,  w = sigmoid(z).
+ * lambda_r: [3 hidden + 1] = v1[hidden], c1[hidden], v2[hidden], c2; 1 <= hidden <= 256.  (The paper says
+ * "2-layer MLP" only; ReLU hidden units and a sigmoid output are this library's reading.)
+ * loss_plus, loss_minus: [B] per-sample losses at theta+ and theta- (the loss outputs of sama_step or
+ * sama_fd_metagrad).  loss_diff: [B] loss_plus - loss_minus as the forward pass formed it (sama_ctx_loss_diff), or
+ * NULL.  Give it whenever it is available: each fp32 loss carries a rounding of about 1e-7 of its size, which
+ * for a small perturbation (alpha = 1e-2) is several 1e-3 of the difference; with loss_diff, loss_plus is
+ * rebuilt as loss_minus + loss_diff and may be NULL.  eps_fd: one float on the device (NULL: the context's).
+ * B_norm: the 1/B of the objective (pass B).  metagrad_r_out: [3 hidden + 1],
+ *   metagrad_r = -[dL_base(theta+)/dlambda_r - dL_base(theta-)/dlambda_r] / (2 eps_fd),
+ * all zero when eps_fd is 0.  This is the vector a data-parallel run would all-reduce once per meta step
+ * (Sec. 3.3).  Accumulated in double in a fixed order: bitwise reproducible.  Needs a context created
+ * with an mlp (for its workspace); B <= max_batch. */
+int sama_fd_metagrad_reweight(sama_ctx* ctx, int32_t B, const float* loss_plus, const float* loss_minus,
+                              const float* loss_diff, int32_t hidden, const float* lambda_r, const float* eps_fd,
+                              int32_t B_norm, float* metagrad_r_out, void* stream);
+
+/* The step of Fig. 2 with the shared reweighting network as the meta learner: sama_adapt -> sama_perturb
+ * -> dual forward pass -> sama_fd_metagrad_reweight, one stream, no host synchronisation.  Arguments as
+ * sama_step, with (hidden, lambda_r, metagrad_r_out) in place of (lambda, metagrad_out). */
+int sama_step_reweight(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* theta, const float* m,
+                       const float* s, const float* g_base, const float* g_meta, const sama_adam_t* adam,
+                       float alpha, const float* X, const int32_t* y, int32_t B, int32_t hidden,
+                       const float* lambda_r, float* p_out, float* theta_plus, float* theta_minus,
+                       float* metagrad_r_out, float* loss_plus_out, float* loss_minus_out, void* stream);
+
+/* SAMA on the biased-regression problem of Appendix E,
+ *   L_meta(w) = ||X' w - y'||^2,   L_base(w, lambda) = ||X w - y||^2 + beta ||w - lambda||^2,
+ * whose meta parameter lambda has the dimension d of w.
+ *
+ * sama_biasreg_direct_grad: the direct gradient of Eq. 1, g_meta = dL_meta/dw = 2 X'^T (X' w - y').
+ * Xv: [n_val][d] row-major, yv: [n_val], w: [d], g_meta_out: [d] (must not overlap the inputs),
+ * meta_loss_out: one float on the device (L_meta(w)) or NULL.  Accumulated in double in a fixed order.
+ * Allocates a workspace inside the context on the first call and when d grows (cudaMalloc; synchronises).
+ *
+ * sama_biasreg_fd_metagrad: Eq. 5 for this objective.  With g_lambda(w) = dL_base/dlambda = -2 beta (w - lambda),
+ *   metagrad = -[g_lambda(w_plus) - g_lambda(w_minus)] / (2 eps_fd)      (all [d]; 0 when eps_fd is 0).
+ * eps_fd: one float on the device (NULL: the context's, as left by sama_perturb).
+ *
+ * sama_biasreg_step: direct gradient -> sama_adapt -> sama_perturb -> sama_biasreg_fd_metagrad on one stream.
+ * An SGD base optimiser is adam->identity = 1 (m, s, g_base may then be NULL).  Outputs g_meta_out, p_out,
+ * w_plus, w_minus, metagrad_out: [d] each, pairwise distinct (p_out may alias g_meta_out). */
+int sama_biasreg_direct_grad(sama_ctx* ctx, int32_t d, int32_t n_val, const float* Xv, const float* yv,
+                             const float* w, float* g_meta_out, float* meta_loss_out, void* stream);
+int sama_biasreg_fd_metagrad(sama_ctx* ctx, int64_t d, const float* w_plus, const float* w_minus,
+                             const float* lambda, float beta, const float* eps_fd, float* metagrad_out,
+                             void* stream);
+int sama_biasreg_step(sama_ctx* ctx, int32_t d, int32_t n_val, const float* Xv, const float* yv, const float* w,
+                      const float* lambda, float beta, const float* m, const float* s, const float* g_base,
+                      const sama_adam_t* adam, float alpha, float* g_meta_out, float* p_out, float* w_plus,
+                      float* w_minus, float* metagrad_out, void* stream);
 
 /* sama_step (Fig. 2) for callers whose data lives in HOST memory: every
  * pointer below is a host pointer (pinned memory makes the copies
@@ -200,6 +261,11 @@ int sama_step_host(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float*
  * eps_fd), valid until sama_destroy. */
 double* sama_ctx_sumsq(sama_ctx* ctx);
 float* sama_ctx_eps_fd(sama_ctx* ctx);
+
+/* Device address of the context's [max_batch] buffer that every forward pass through this context
+ * (sama_fd_metagrad, sama_step, ...) fills with loss+_i - loss-_i, formed inside its last kernel before
+ * either loss is rounded to fp32.  NULL for a context created without an mlp.  Valid until sama_destroy. */
+float* sama_ctx_loss_diff(sama_ctx* ctx);
 
 /* Synchronises `stream`, returns the OR of the device status bits raised since
  * the last call in *status_out and clears them. */
@@ -220,6 +286,12 @@ const char* sama_status_string(int status);
  * to fp32).  Returns SAMA_ERR_UNSUPPORTED for a mode this build lacks. */
 int sama_set_gemm_mode(sama_ctx* ctx, int mode);
 
+/* How the last forward pass run through this context (sama_fd_metagrad, sama_step, sama_step_host)
+ * multiplied matrices: 0 = none yet, 1 = fp32 FMA on the CUDA cores, 2 = tensor cores (3xTF32).  In
+ * automatic mode a model that does not fit the operand workspace sized at sama_create takes path 1,
+ * which is several times slower; this query makes that visible. */
+int sama_last_forward_path(sama_ctx* ctx);
+
 /* Number of kernels the library has launched through this context. */
 int64_t sama_launch_count(sama_ctx* ctx);
 
@@ -239,15 +311,23 @@ enum {
     SAMA_K_HEAD = 7, /* narrow last layer fused with cross-entropy + central difference */
     SAMA_K_PERTURB_SPLIT = 8, /* perturbation that also writes the tensor-core operands of W+ and W- */
     SAMA_K_META_GEMM = 9,     /* matrix products of the direct gradient (forward, dz W, dz^T h) */
-    SAMA_K_META_AUX = 10      /* softmax gradient, bias sums, mean loss of the direct gradient */
+    SAMA_K_META_AUX = 10,     /* softmax gradient, bias sums, mean loss of the direct gradient */
+    SAMA_K_REWEIGHT_FD = 11,  /* central difference of the shared reweighting network's gradient (Eq. 5, Sec. 4.1) */
+    SAMA_K_BIASREG_GRAD = 12, /* direct gradient of the biased-regression meta objective (Appendix E) */
+    SAMA_K_BIASREG_FD = 13,   /* central difference for the biased-regression base objective */
+    SAMA_K_FUSED_SWEEP = 14   /* adaptation + norm + perturbation + operand split in one launch (small models) */
 };
 typedef struct sama_kernel_time_t {
-    int32_t kind;  /* SAMA_K_* */
-    int32_t layer; /* layer index for the forward kernels, else -1 */
-    float ms;      /* device time between the two events */
+    int32_t kind;     /* SAMA_K_* */
+    int32_t layer;    /* layer index for the forward kernels, else -1 */
+    float ms;         /* device time between the two events */
+    int32_t launches; /* launches between the two events: 1, or the length of a run in grouped mode */
 } sama_kernel_time_t;
 
-/* on != 0: start recording (discarding earlier records); on == 0: stop and discard. */
+/* on == 1: start recording, one event pair per launch (discarding earlier records).  on == 2: grouped --
+ * consecutive launches of the same kind (the layers of one forward pass) share one event pair, so no event
+ * sits between them and they overlap as they do in an untimed step (programmatic dependent launch).
+ * on == 0: stop and discard. */
 int sama_profile_enable(sama_ctx* ctx, int32_t on);
 
 /* Waits for the recorded events, writes up to `capacity` records (launch

@@ -43,11 +43,12 @@ class sama_adam_t(C.Structure):
 
 
 class sama_kernel_time_t(C.Structure):
-    _fields_ = [("kind", C.c_int32), ("layer", C.c_int32), ("ms", C.c_float)]
+    _fields_ = [("kind", C.c_int32), ("layer", C.c_int32), ("ms", C.c_float), ("launches", C.c_int32)]
 
 
 KERNEL_KINDS = {0: "adapt_sumsq", 1: "sumsq", 2: "perturb", 3: "gemm_ffma", 4: "ce_fd", 5: "split_tf32",
-                6: "gemm_tf32x3", 7: "head_ce_fd", 8: "perturb_split", 9: "meta_gemm", 10: "meta_aux"}
+                6: "gemm_tf32x3", 7: "head_ce_fd", 8: "perturb_split", 9: "meta_gemm", 10: "meta_aux",
+                11: "reweight_fd", 12: "biasreg_grad", 13: "biasreg_fd", 14: "fused_sweep"}
 
 
 class sama_mlp_t(C.Structure):
@@ -92,6 +93,16 @@ lib.sama_fd_metagrad.argtypes = [_vp, C.POINTER(sama_mlp_t), _vp, _vp, _vp, _vp,
                                  _vp, _vp]
 lib.sama_step.argtypes = [_vp, C.POINTER(sama_mlp_t), C.c_int64, _vp, _vp, _vp, _vp, _vp, C.POINTER(sama_adam_t),
                           C.c_float, _vp, _vp, _vp, C.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.sama_fd_metagrad_reweight.argtypes = [_vp, C.c_int32, _vp, _vp, _vp, C.c_int32, _vp, _vp, C.c_int32, _vp, _vp]
+lib.sama_ctx_loss_diff.argtypes = [_vp]
+lib.sama_ctx_loss_diff.restype = _vp
+lib.sama_step_reweight.argtypes = [_vp, C.POINTER(sama_mlp_t), C.c_int64, _vp, _vp, _vp, _vp, _vp,
+                                   C.POINTER(sama_adam_t), C.c_float, _vp, _vp, C.c_int32, C.c_int32, _vp, _vp, _vp,
+                                   _vp, _vp, _vp, _vp, _vp]
+lib.sama_biasreg_direct_grad.argtypes = [_vp, C.c_int32, C.c_int32, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.sama_biasreg_fd_metagrad.argtypes = [_vp, C.c_int64, _vp, _vp, _vp, C.c_float, _vp, _vp, _vp]
+lib.sama_biasreg_step.argtypes = [_vp, C.c_int32, C.c_int32, _vp, _vp, _vp, _vp, C.c_float, _vp, _vp, _vp,
+                                  C.POINTER(sama_adam_t), C.c_float, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.sama_meta_grad.argtypes = [_vp, C.POINTER(sama_mlp_t), _vp, _vp, _vp, C.c_int32, _vp, _vp, _vp]
 lib.sama_step_host.argtypes = [_vp, C.POINTER(sama_mlp_t), C.c_int64, _vp, _vp, _vp, _vp, _vp,
                                C.POINTER(sama_adam_t), C.c_float, _vp, _vp, _vp, C.c_int32, _vp, _vp, _vp, _vp]
@@ -107,6 +118,7 @@ lib.sama_status_string.argtypes = [C.c_int]
 lib.sama_status_string.restype = C.c_char_p
 lib.sama_set_gemm_mode.argtypes = [_vp, C.c_int]
 lib.sama_launch_count.argtypes = [_vp]
+lib.sama_last_forward_path.argtypes = [_vp]
 lib.sama_launch_count.restype = C.c_int64
 lib.sama_profile_enable.argtypes = [_vp, C.c_int32]
 lib.sama_profile_collect.argtypes = [_vp, C.POINTER(sama_kernel_time_t), C.c_int32, C.POINTER(C.c_int32)]
@@ -193,6 +205,50 @@ def sama_step(ctx, mlp: MLP, n, theta, m, s, g_base, g_meta, adam: Adam, alpha, 
                                 _ptr(loss_minus_out), _stream(stream)), "sama_step")
 
 
+def sama_ctx_loss_diff(ctx) -> int:
+    return lib.sama_ctx_loss_diff(ctx)
+
+
+def sama_fd_metagrad_reweight(ctx, B, loss_plus, loss_minus, loss_diff, hidden, lambda_r, eps_fd, B_norm,
+                              metagrad_r_out, stream=None) -> int:
+    return _check(lib.sama_fd_metagrad_reweight(ctx, int(B), _ptr(loss_plus), _ptr(loss_minus), _ptr(loss_diff),
+                                                int(hidden),
+                                                _ptr(lambda_r), _ptr(eps_fd), int(B_norm), _ptr(metagrad_r_out),
+                                                _stream(stream)), "sama_fd_metagrad_reweight")
+
+
+def sama_step_reweight(ctx, mlp: MLP, n, theta, m, s, g_base, g_meta, adam: Adam, alpha, X, y, B, hidden, lambda_r,
+                       p_out, theta_plus, theta_minus, metagrad_r_out, loss_plus_out=None, loss_minus_out=None,
+                       stream=None) -> int:
+    a = adam.c()
+    return _check(lib.sama_step_reweight(ctx, mlp.c(), int(n), _ptr(theta), _ptr(m), _ptr(s), _ptr(g_base),
+                                         _ptr(g_meta), C.byref(a), float(alpha), _ptr(X), _ptr(y), int(B),
+                                         int(hidden), _ptr(lambda_r), _ptr(p_out), _ptr(theta_plus),
+                                         _ptr(theta_minus), _ptr(metagrad_r_out), _ptr(loss_plus_out),
+                                         _ptr(loss_minus_out), _stream(stream)), "sama_step_reweight")
+
+
+def sama_biasreg_direct_grad(ctx, d, n_val, Xv, yv, w, g_meta_out, meta_loss_out=None, stream=None) -> int:
+    return _check(lib.sama_biasreg_direct_grad(ctx, int(d), int(n_val), _ptr(Xv), _ptr(yv), _ptr(w),
+                                               _ptr(g_meta_out), _ptr(meta_loss_out), _stream(stream)),
+                  "sama_biasreg_direct_grad")
+
+
+def sama_biasreg_fd_metagrad(ctx, d, w_plus, w_minus, lam, beta, eps_fd, metagrad_out, stream=None) -> int:
+    return _check(lib.sama_biasreg_fd_metagrad(ctx, int(d), _ptr(w_plus), _ptr(w_minus), _ptr(lam), float(beta),
+                                               _ptr(eps_fd), _ptr(metagrad_out), _stream(stream)),
+                  "sama_biasreg_fd_metagrad")
+
+
+def sama_biasreg_step(ctx, d, n_val, Xv, yv, w, lam, beta, m, s, g_base, adam: Adam, alpha, g_meta_out, p_out,
+                      w_plus, w_minus, metagrad_out, stream=None) -> int:
+    a = adam.c()
+    return _check(lib.sama_biasreg_step(ctx, int(d), int(n_val), _ptr(Xv), _ptr(yv), _ptr(w), _ptr(lam), float(beta),
+                                        _ptr(m), _ptr(s), _ptr(g_base), C.byref(a), float(alpha), _ptr(g_meta_out),
+                                        _ptr(p_out), _ptr(w_plus), _ptr(w_minus), _ptr(metagrad_out),
+                                        _stream(stream)), "sama_biasreg_step")
+
+
 def sama_meta_grad(ctx, mlp: MLP, theta, X_meta, y_meta, B, g_meta_out, loss_out=None, stream=None) -> int:
     return _check(lib.sama_meta_grad(ctx, mlp.c(), _ptr(theta), _ptr(X_meta), _ptr(y_meta), int(B),
                                      _ptr(g_meta_out), _ptr(loss_out), _stream(stream)), "sama_meta_grad")
@@ -235,13 +291,20 @@ def sama_launch_count(ctx) -> int:
     return int(lib.sama_launch_count(ctx))
 
 
-def sama_profile_enable(ctx, on: bool) -> int:
-    return _check(lib.sama_profile_enable(ctx, int(bool(on))), "sama_profile_enable")
+def sama_last_forward_path(ctx) -> int:
+    return int(lib.sama_last_forward_path(ctx))
 
 
-def sama_profile_collect(ctx, capacity: int = 65536):
-    """Returns [(kind, layer, ms), ...] in launch order."""
+def sama_profile_enable(ctx, on) -> int:
+    """on: 0 / False = off, 1 / True = one event pair per launch, 2 = one pair per run of same-kind launches."""
+    return _check(lib.sama_profile_enable(ctx, int(on)), "sama_profile_enable")
+
+
+def sama_profile_collect(ctx, capacity: int = 65536, with_launches: bool = False):
+    """Returns [(kind, layer, ms), ...] in launch order ((kind, layer, ms, launches) with ``with_launches``)."""
     buf = (sama_kernel_time_t * capacity)()
     cnt = C.c_int32(0)
     _check(lib.sama_profile_collect(ctx, buf, capacity, C.byref(cnt)), "sama_profile_collect")
+    if with_launches:
+        return [(buf[i].kind, buf[i].layer, buf[i].ms, buf[i].launches) for i in range(cnt.value)]
     return [(buf[i].kind, buf[i].layer, buf[i].ms) for i in range(cnt.value)]

@@ -1,0 +1,138 @@
+// SAMA on the biased-regression problem of Appendix E:
+//   L_meta(w)         = || X' w - y' ||^2
+//   L_base(w, lambda) = || X w - y ||^2 + beta || w - lambda ||^2
+// Two kernels, both specific to this objective; adaptation, norm and perturbation are the library's own.
+//
+//   direct gradient (Eq. 1):  g_meta = dL_meta/dw = 2 X'^T (X' w - y')
+//   central difference (Eq. 5) of g_lambda(w) = dL_base/dlambda = -2 beta (w - lambda):
+//                             metagrad = -[g_lambda(w+) - g_lambda(w-)] / (2 eps_fd)
+//
+// The direct gradient reads X' once from HBM: a block takes a contiguous run of rows, eight at a time; each warp
+// forms one residual r_i = x_i . w - y_i, then all threads add r_i x_i into the block's partial gradient in
+// shared memory (the rows come back from L1 / L2).  Blocks are added in block order by the last block to
+// arrive.  Accumulation is double throughout; nothing depends on scheduling.
+#include "sama_internal.h"
+
+namespace sama {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kRows = kThreads / 32;  // rows in flight per block = warps
+
+__global__ void __launch_bounds__(kThreads)
+biasreg_direct_grad_kernel(int d, int n_val, const float* __restrict__ Xv, const float* __restrict__ yv,
+                           const float* __restrict__ w, float* __restrict__ g_out, float* __restrict__ loss_out,
+                           double* partials, DeviceScalars* sc) {
+    extern __shared__ double g_s[];        // [d] partial gradient, then [kRows] residuals
+    double* r_s = g_s + d;
+    __shared__ bool is_last;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int c = threadIdx.x; c < d; c += kThreads) g_s[c] = 0.0;
+    // this block's rows: a contiguous run, the same for every launch of this shape
+    const int per = (n_val + gridDim.x - 1) / gridDim.x;
+    const int row0 = blockIdx.x * per, row1 = min(n_val, row0 + per);
+    double sq = 0.0;                        // sum of r_i^2 over this block's rows (thread 0 of each warp)
+    __syncthreads();
+    for (int base = row0; base < row1; base += kRows) {
+        const int i = base + warp;
+        double r = 0.0;
+        if (i < row1) {
+            const float* x = Xv + (int64_t)i * d;
+            for (int c = lane; c < d; c += 32) r = fma((double)x[c], (double)w[c], r);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) r += __shfl_xor_sync(0xffffffffu, r, o);
+            r -= (double)yv[i];
+            if (lane == 0) sq += r * r;
+        }
+        if (lane == 0) r_s[warp] = (i < row1) ? r : 0.0;
+        __syncthreads();
+        const int rows = min(kRows, row1 - base);
+        for (int c = threadIdx.x; c < d; c += kThreads) {
+            double a = g_s[c];
+            for (int k = 0; k < rows; ++k) a = fma((double)Xv[(int64_t)(base + k) * d + c], r_s[k], a);
+            g_s[c] = a;
+        }
+        __syncthreads();
+    }
+    double* mine = partials + (size_t)blockIdx.x * (d + 1);
+    for (int c = threadIdx.x; c < d; c += kThreads) mine[c] = g_s[c];
+    // the block's share of the meta loss: warps in order
+    if (lane == 0) r_s[warp] = sq;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int k = 0; k < kRows; ++k) t += r_s[k];
+        mine[d] = t;
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned prev = atomicAdd(&sc->counter, 1u);
+        is_last = (prev == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    for (int c = threadIdx.x; c <= d; c += kThreads) {
+        double t = 0.0;
+        for (unsigned b = 0; b < gridDim.x; ++b) t += __ldcg(partials + (size_t)b * (d + 1) + c);
+        if (c < d) g_out[c] = (float)(2.0 * t);
+        else if (loss_out) *loss_out = (float)t;
+    }
+    if (threadIdx.x == 0) sc->counter = 0u;
+}
+
+__global__ void __launch_bounds__(kThreads)
+biasreg_fd_kernel(int64_t d, const float* __restrict__ w_plus, const float* __restrict__ w_minus,
+                  const float* __restrict__ lambda, float beta, const float* __restrict__ eps_fd,
+                  float* __restrict__ out) {
+    pdl_trigger();
+    pdl_wait();
+    // double: w+- - lambda is then exact, so the only rounding the quotient amplifies is that of w+- themselves
+    const double eps = (double)*eps_fd;
+    const double inv = eps > 0.0 ? 1.0 / (2.0 * eps) : 0.0;
+    const double b2 = 2.0 * (double)beta;
+    const int64_t stride = (int64_t)gridDim.x * kThreads;
+    for (int64_t k = (int64_t)blockIdx.x * kThreads + threadIdx.x; k < d; k += stride) {
+        const double lam = (double)lambda[k];
+        const double gp = -b2 * ((double)w_plus[k] - lam);    // dL_base/dlambda at w+
+        const double gm = -b2 * ((double)w_minus[k] - lam);   // ... at w-
+        out[k] = (float)(-(gp - gm) * inv);
+    }
+}
+
+}  // namespace
+
+int biasreg_grid(const sama_ctx* ctx, int n_val) {
+    int g = (n_val + kRows - 1) / kRows;
+    if (g > ctx->sm_count) g = ctx->sm_count;
+    return g < 1 ? 1 : g;
+}
+
+cudaError_t launch_biasreg_direct_grad(sama_ctx* ctx, int d, int n_val, const float* Xv, const float* yv,
+                                       const float* w, float* g_out, float* loss_out, cudaStream_t st) {
+    const size_t smem = sizeof(double) * ((size_t)d + kRows);
+    if (smem > 48 * 1024) {
+        const cudaError_t e = cudaFuncSetAttribute(biasreg_direct_grad_kernel,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    KernelScope scope(ctx, SAMA_K_BIASREG_GRAD, -1, st);
+    biasreg_direct_grad_kernel<<<biasreg_grid(ctx, n_val), kThreads, smem, st>>>(d, n_val, Xv, yv, w, g_out, loss_out,
+                                                                                 ctx->br_partials, ctx->scalars);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_biasreg_fd(sama_ctx* ctx, int64_t d, const float* w_plus, const float* w_minus,
+                              const float* lambda, float beta, const float* eps_fd, float* out, cudaStream_t st) {
+    int64_t blocks = (d + kThreads - 1) / kThreads;
+    const int64_t cap = (int64_t)ctx->sm_count * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    KernelScope scope(ctx, SAMA_K_BIASREG_FD, -1, st);
+    return launch_dependent(biasreg_fd_kernel, dim3((unsigned)blocks), dim3(kThreads), 0, st, d, w_plus, w_minus, lambda,
+                            beta, eps_fd, out);
+}
+
+}  // namespace sama

@@ -38,7 +38,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 ce_fd_kernel(const float* __restrict__ zp, const float* __restrict__ zm, int ldz, const int32_t* __restrict__ y,
              const float* __restrict__ lambda, int B, int C, const float* __restrict__ eps_fd,
              float* __restrict__ metagrad, float* __restrict__ loss_plus, float* __restrict__ loss_minus,
-             DeviceScalars* sc) {
+             float* __restrict__ loss_diff, DeviceScalars* sc) {
     pdl_trigger();
     pdl_wait();
     const int lane = threadIdx.x & 31;
@@ -56,9 +56,12 @@ ce_fd_kernel(const float* __restrict__ zp, const float* __restrict__ zm, int ldz
     if (loss_plus) loss_plus[i] = lse_p - zyp;
     if (loss_minus) loss_minus[i] = lse_m - zym;
     const float eps = *eps_fd;
+    const float d = (lse_p - lse_m) - (zyp - zym);
+    // loss+ - loss- as formed here, i.e. without the rounding of the two losses to fp32 (which is of the order
+    // of the difference itself when the perturbation is small)
+    if (loss_diff) loss_diff[i] = ok ? d : 0.f;
     float out = 0.f;
     if (ok && eps > 0.f) {
-        const float d = (lse_p - lse_m) - (zyp - zym);
         const float sg = 1.0f / (1.0f + expf(-lambda[i]));
         out = -(sg * (1.0f - sg)) * d / (2.0f * eps * (float)B);
     }
@@ -69,11 +72,11 @@ ce_fd_kernel(const float* __restrict__ zp, const float* __restrict__ zm, int ldz
 
 cudaError_t launch_ce_fd(sama_ctx* ctx, const float* z_plus, const float* z_minus, int ldz, const int32_t* y,
                          const float* lambda, int B, int C, const float* eps_fd, float* metagrad,
-                         float* loss_plus, float* loss_minus, cudaStream_t st) {
+                         float* loss_plus, float* loss_minus, float* loss_diff, cudaStream_t st) {
     const int grid = (B + kWarpsPerBlock - 1) / kWarpsPerBlock;
     KernelScope scope(ctx, SAMA_K_CE_FD, -1, st);
     return launch_dependent(ce_fd_kernel, dim3(grid), dim3(kWarpsPerBlock * 32), 0, st, z_plus, z_minus, ldz, y, lambda,
-                            B, C, eps_fd, metagrad, loss_plus, loss_minus, ctx->scalars);
+                            B, C, eps_fd, metagrad, loss_plus, loss_minus, loss_diff, ctx->scalars);
 }
 
 }  // namespace sama

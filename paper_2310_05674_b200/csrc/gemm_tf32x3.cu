@@ -38,6 +38,7 @@
 #include <cuda.h>
 
 #include <cstdlib>
+#include <new>
 
 #include "sama_internal.h"
 
@@ -245,8 +246,18 @@ __device__ __forceinline__ float to_tf32(float x) {
 // Round-to-nearest (ties away from zero) to TF32 with integer arithmetic: same result as cvt.rna.tf32.f32 on
 // finite values, at the full integer rate (the conversion instruction issues at a fraction of it, which shows
 // in the epilogue, where eight warps convert a whole tile).
+// NaN and infinity (exponent field all ones) pass through unchanged: the add could otherwise carry a NaN's
+// mantissa into the sign bit and turn it into a zero.
 __device__ __forceinline__ float round_tf32(float x) {
-    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);
+    const uint32_t u = __float_as_uint(x);
+    const uint32_t r = (u + 0x1000u) & 0xFFFFE000u;
+    return __uint_as_float((u & 0x7F800000u) == 0x7F800000u ? u : r);
+}
+// Bias, then ReLU as a select that keeps NaN (max(NaN, 0) would return 0 and hide a non-finite input):
+// floor_v is 0 for ReLU and -infinity (never below) otherwise.
+__device__ __forceinline__ float bias_act(float x, float b, float floor_v) {
+    const float v = x + b;
+    return v < floor_v ? 0.f : v;
 }
 
 struct TcArgs {
@@ -309,13 +320,13 @@ __device__ __forceinline__ void store_block(const TcArgs& args, const float4* st
     float4 t[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) t[i] = ((i & 1) ? src_odd : src_even)[(i >> 1) * 64];
-    const float floor_v = relu ? 0.f : -3.402823466e38f;  // max(x, floor_v): ReLU or (for finite x) nothing
+    const float floor_v = relu ? 0.f : -INFINITY;  // values below floor_v become 0: ReLU, or nothing
     if (full && rows == 32 && mk == nullptr && (vec_f32 || !want_f32)) {
         // interior block: no per-row or per-column conditions (branches cost more here than the arithmetic)
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            const float v0 = fmaxf(t[i].x + b[0], floor_v), v1 = fmaxf(t[i].y + b[1], floor_v);
-            const float v2 = fmaxf(t[i].z + b[2], floor_v), v3 = fmaxf(t[i].w + b[3], floor_v);
+            const float v0 = bias_act(t[i].x, b[0], floor_v), v1 = bias_act(t[i].y, b[1], floor_v);
+            const float v2 = bias_act(t[i].z, b[2], floor_v), v3 = bias_act(t[i].w, b[3], floor_v);
             if (want_f32) *reinterpret_cast<float4*>(dst + i * dst_step) = make_float4(v0, v1, v2, v3);
             if (want_split) {
                 const float h0 = round_tf32(v0), h1 = round_tf32(v1), h2 = round_tf32(v2), h3 = round_tf32(v3);
@@ -331,8 +342,8 @@ __device__ __forceinline__ void store_block(const TcArgs& args, const float4* st
         const int rl = r0 + 4 * i;
         if (rl < rows) {
             const float4 ti = ((i & 1) ? src_odd : src_even)[(i >> 1) * 64];
-            float v[4] = {fmaxf(ti.x + b[0], floor_v), fmaxf(ti.y + b[1], floor_v), fmaxf(ti.z + b[2], floor_v),
-                          fmaxf(ti.w + b[3], floor_v)};
+            float v[4] = {bias_act(ti.x, b[0], floor_v), bias_act(ti.y, b[1], floor_v), bias_act(ti.z, b[2], floor_v),
+                          bias_act(ti.w, b[3], floor_v)};
             if (mk) {  // backward pass: the derivative passes only where the forward activation was positive
                 const float* mrow = mk + i * mk_step;
 #pragma unroll
@@ -921,41 +932,70 @@ bool make_map(CUtensorMap* map, const float* base, int ld, int64_t rows, int sla
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Per-context state of the tensor-core path, set up once by tc_state_create on the context's device:
+// experiment switches (environment variables read once), how many CTA pairs the cluster scheduler can keep
+// resident, and a cache of encoded tensor maps, so that a warm launch path neither reads the environment nor
+// calls into the driver.
+struct TcMapKey {
+    const void* base;
+    int64_t rows, slab;
+    int ld, slabs, box_rows;
+    bool operator==(const TcMapKey& o) const {
+        return base == o.base && rows == o.rows && slab == o.slab && ld == o.ld && slabs == o.slabs &&
+               box_rows == o.box_rows;
+    }
+};
+struct TcState {
+    int tile = 0;          // SAMA_TC_TILE: 64 / 128 force a single-CTA tile width, 256 the CTA pair
+    bool no_pair = false;  // SAMA_TC_PAIR=0
+    bool no_ksplit = false;  // SAMA_TC_KSPLIT=1
+    bool no_tail = false;  // SAMA_TC_TAIL=0
+    int group = 0;         // SAMA_TC_GROUP
+    int pair_units = 0;    // co-resident CTA pairs of the 256 x 256 kernel on this device
+    static constexpr int kCache = 64;
+    TcMapKey keys[kCache];
+    CUtensorMap maps[kCache];
+    int n_cached = 0, next_victim = 0;
+};
+inline TcState* tc_state(sama_ctx* ctx) { return static_cast<TcState*>(ctx->tc_state); }
+
+// The map for `key`, encoded on first use.  nullptr if the driver refuses the encoding.
+const CUtensorMap* cached_map(TcState* st, const float* base, int ld, int64_t rows, int slabs, int box_rows,
+                              int64_t slab) {
+    const TcMapKey key{base, rows, slab, ld, slabs, box_rows};
+    for (int i = 0; i < st->n_cached; ++i)
+        if (st->keys[i] == key) return &st->maps[i];
+    int slot;
+    if (st->n_cached < TcState::kCache) {
+        slot = st->n_cached++;
+    } else {
+        slot = st->next_victim;
+        st->next_victim = (st->next_victim + 1) % TcState::kCache;
+    }
+    if (!make_map(&st->maps[slot], base, ld, rows, slabs, box_rows, slab)) {
+        st->n_cached = 0;  // the slot may hold half an encoding: start over
+        return nullptr;
+    }
+    st->keys[slot] = key;
+    return &st->maps[slot];
+}
+
+template <int BN, bool PAIR, int EPI>
+cudaError_t tc_prepare_kernel() {
+    return cudaFuncSetAttribute(gemm_tf32x3_kernel<BN, PAIR, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                smem_bytes(PAIR ? BN / 2 : BN));
+}
+
 // Launches the persistent kernel on min(work items, co-resident CTAs or CTA pairs) units.
 template <int BN, bool PAIR, int EPI>
-cudaError_t launch_tc(const CUtensorMap maps[4], const TcArgs& a, int items, int sm_count, cudaStream_t st,
-                      size_t ws_floats = 0, int tail_flags = 0) {
+cudaError_t launch_tc(const CUtensorMap* const maps[4], const TcArgs& a, int items, int max_units, bool tail_ok,
+                      cudaStream_t st, size_t ws_floats = 0, int tail_flags = 0) {
     const int ks = PAIR ? 1 : a.ksplit;
     constexpr int kSmem = smem_bytes(PAIR ? BN / 2 : BN);
-    static int max_units = 0;  // one CTA per SM (shared memory); pairs: what the cluster scheduler can co-schedule
-    if (max_units == 0) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tf32x3_kernel<BN, PAIR, EPI>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
-        if (e != cudaSuccess) return e;
-        int units = sm_count;
-        if (PAIR) {
-            cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(2 * (sm_count / 2));
-            cfg.blockDim = dim3(threads_for(EPI));
-            cfg.dynamicSmemBytes = kSmem;
-            cudaLaunchAttribute attr[1];
-            attr[0].id = cudaLaunchAttributeClusterDimension;
-            attr[0].val.clusterDim.x = 2;
-            attr[0].val.clusterDim.y = 1;
-            attr[0].val.clusterDim.z = 1;
-            cfg.attrs = attr;
-            cfg.numAttrs = 1;
-            int clusters = 0;
-            e = cudaOccupancyMaxActiveClusters(&clusters, gemm_tf32x3_kernel<BN, PAIR, EPI>, &cfg);
-            if (e != cudaSuccess) return e;
-            units = clusters < sm_count / 2 ? clusters : sm_count / 2;
-        }
-        if (units < 1) return cudaErrorLaunchOutOfResources;
-        max_units = units;
-    }
+    if (max_units < 1) return cudaErrorLaunchOutOfResources;
     if (ks > 1)  // one tile per cluster of ks CTAs
         return launch_clustered(ks, gemm_tf32x3_kernel<BN, PAIR, EPI>, dim3(items * ks), dim3(threads_for(EPI)),
-                                (size_t)kSmem, st, maps[0], maps[1], maps[2], maps[3], a);
+                                (size_t)kSmem, st, *maps[0], *maps[1], *maps[2], *maps[3], a);
     const int units = items < max_units ? items : max_units;
     TcArgs b = a;
     b.full_rounds = 0;
@@ -964,15 +1004,14 @@ cudaError_t launch_tc(const CUtensorMap maps[4], const TcArgs& a, int items, int
         // tiles that do not fill the last round are each shared by two pairs when that takes no more pairs
         // than there are (and the contraction is long enough to be worth an exchange)
         const int rounds = items / max_units, tail = items % max_units;
-        static const bool off = []() { const char* e = std::getenv("SAMA_TC_TAIL"); return e && e[0] == '0'; }();
-        if (!off && tail > 0 && 2 * tail <= max_units && a.num_kb >= 16 && a.flags && tail * 4 <= tail_flags &&
+        if (tail_ok && tail > 0 && 2 * tail <= max_units && a.num_kb >= 16 && a.flags && tail * 4 <= tail_flags &&
             (size_t)tail * 4 * BM * BN <= ws_floats) {
             b.full_rounds = rounds;
             b.tail_tiles = tail;
         }
     }
     return launch_clustered(PAIR ? 2 : 1, gemm_tf32x3_kernel<BN, PAIR, EPI>, dim3(units * (PAIR ? 2 : 1)),
-                            dim3(threads_for(EPI)), (size_t)kSmem, st, maps[0], maps[1], maps[2], maps[3], b);
+                            dim3(threads_for(EPI)), (size_t)kSmem, st, *maps[0], *maps[1], *maps[2], *maps[3], b);
 }
 
 inline int round_up32(int x) { return (x + 31) & ~31; }
@@ -1011,10 +1050,51 @@ cudaError_t launch_split_transpose_tf32(sama_ctx* ctx, const float* src, int64_t
     return launch_dependent(split_transpose_tf32_kernel, grid, dim3(256), 0, st, src, rows, cols, ld_out, hi, lo);
 }
 
+// Set-up of the tensor-core path for a context (called by sama_create with the context's device current):
+// reads the experiment switches, opts every kernel instantiation into its shared-memory size on this
+// device, and asks how many CTA pairs can be resident.
+cudaError_t tc_state_create(sama_ctx* ctx) {
+    TcState* st = new (std::nothrow) TcState();
+    if (!st) return cudaErrorMemoryAllocation;
+    ctx->tc_state = st;
+    if (const char* e = std::getenv("SAMA_TC_TILE")) st->tile = std::atoi(e);
+    if (const char* e = std::getenv("SAMA_TC_PAIR")) st->no_pair = std::atoi(e) == 0;
+    if (const char* e = std::getenv("SAMA_TC_KSPLIT")) st->no_ksplit = std::atoi(e) == 1;
+    if (const char* e = std::getenv("SAMA_TC_TAIL")) st->no_tail = e[0] == '0';
+    if (const char* e = std::getenv("SAMA_TC_GROUP")) st->group = std::atoi(e);
+    cudaError_t e;
+    if ((e = tc_prepare_kernel<256, true, 8>()) != cudaSuccess) return e;
+    if ((e = tc_prepare_kernel<128, false, 8>()) != cudaSuccess) return e;
+    if ((e = tc_prepare_kernel<64, false, 8>()) != cudaSuccess) return e;
+    if ((e = tc_prepare_kernel<16, false, 4>()) != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (ctx->sm_count / 2));
+    cfg.blockDim = dim3(threads_for(8));
+    cfg.dynamicSmemBytes = smem_bytes(128);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    if ((e = cudaOccupancyMaxActiveClusters(&clusters, gemm_tf32x3_kernel<256, true, 8>, &cfg)) != cudaSuccess) return e;
+    st->pair_units = clusters < ctx->sm_count / 2 ? clusters : ctx->sm_count / 2;
+    return cudaSuccess;
+}
+
+void tc_state_destroy(sama_ctx* ctx) {
+    delete tc_state(ctx);
+    ctx->tc_state = nullptr;
+}
+
 // One layer on the tensor cores.  a_hi/a_lo: [shared_a ? 1 : 2][M][Kp]; w_hi/w_lo: [2][N][Kp]; Kp = K rounded
 // up to 32.  Hidden layers write the next operands (out_hi/out_lo, [2][M][round_up32(N)]); the last layer
 // writes fp32 logits.
 cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st) {
+    TcState* ts = tc_state(ctx);
+    if (!ts) return cudaErrorInvalidValue;
     const int Kp = round_up32(L.K);
     const int nbr = L.branches == 1 ? 1 : 2;  // the direct gradient runs a single branch
     const int num_kb = Kp / BKF;
@@ -1022,7 +1102,8 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     // write the zero padding up to round_up32(N)).  Otherwise the candidates are single-CTA tiles of 128 x 64
     // and 128 x 128 and the CTA pair's 256 x 256; the one with the lowest estimate of
     //   rounds x (k-blocks x time per k-block + time to store a tile),  rounds = ceil(tiles / co-resident units)
-    // is taken.  Times per k-block (microseconds, measured on the three workloads): wider tiles do more
+    // is taken (a pair kernel whose last round is shared by two pairs per tile counts that round as half).
+    // Times per k-block (microseconds, measured on the three workloads): wider tiles do more
     // work per staged operand byte, narrower ones fill the machine when the layer has few tiles.
     const bool narrow_last = L.last && L.N <= 16;
     int bn = 64, ksplit = 1;
@@ -1032,17 +1113,20 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     } else {
         struct Cand { int bn; bool pair; double t_kb, t_tile; };
         const Cand cands[3] = {{64, false, 0.55, 3.0}, {128, false, 0.72, 4.0}, {256, true, 1.12, 6.0}};
-        const bool pair_ok = L.M > BM && L.N >= 256;
-        bool no_pair = false;
-        if (const char* e = std::getenv("SAMA_TC_PAIR")) no_pair = std::atoi(e) == 0;
+        const bool pair_ok = L.M > BM && L.N >= 256 && ts->pair_units > 0;
+        const bool no_pair = ts->no_pair;
         double best = 0.0;
         for (const Cand& c : cands) {
             if (c.bn == 128 && L.N <= 64) continue;
             if (c.pair && (!pair_ok || no_pair)) continue;
             const int64_t tm = c.pair ? (L.M + 2 * BM - 1) / (2 * BM) : (L.M + BM - 1) / BM;
             const int64_t items = tm * ((L.N + c.bn - 1) / c.bn) * nbr;
-            const int64_t units = c.pair ? ctx->sm_count / 2 : ctx->sm_count;
-            const double cost = (double)((items + units - 1) / units) * (num_kb * c.t_kb + c.t_tile);
+            const int64_t units = c.pair ? ts->pair_units : ctx->sm_count;
+            double rounds = (double)((items + units - 1) / units);
+            if (c.pair && !ts->no_tail && items > units && items % units > 0 && 2 * (items % units) <= units &&
+                num_kb >= 16)
+                rounds = (double)(items / units) + 0.55;
+            const double cost = rounds * (num_kb * c.t_kb + c.t_tile);
             if (best == 0.0 || cost < best) { best = cost; bn = c.bn; pair = c.pair; ksplit = 1; }
             // a layer with few tiles: a cluster of 2 or 4 CTAs shares each tile's contraction (one wave,
             // at least two k-blocks per CTA, about 4 us for the exchange; each CTA stores 1 / ks of the tile)
@@ -1054,24 +1138,23 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
                 if (cost_ks < best) { best = cost_ks; bn = c.bn; pair = false; ksplit = ks; }
             }
         }
-        if (const char* e = std::getenv("SAMA_TC_KSPLIT")) { if (std::atoi(e) == 1) ksplit = 1; }
-        // override for experiments (SAMA_TC_TILE): 64 / 128 force a single-CTA width, 256 the pair
-        const int ov = ctx->tile_override;
+        if (ts->no_ksplit) ksplit = 1;
+        // overrides for experiments (SAMA_TC_TILE): 64 / 128 force a single-CTA width, 256 the pair
+        const int ov = ts->tile;
         if (ov == 64 || ov == 128) { bn = ov; pair = false; ksplit = 1; }
         if (ov == 256 && pair_ok && !no_pair) { bn = 256; pair = true; ksplit = 1; }
     }
-    CUtensorMap maps[4];
     const int a_slabs = (L.shared_a || nbr == 1) ? 1 : 2;
     // a box never exceeds the tensor's extent; rows of the shared-memory tile that no copy fills only
     // feed output rows / columns that the epilogue does not store
     const int wrows = pair ? bn / 2 : bn;
     const int a_box = L.M < BM ? L.M : BM, w_box = L.N < wrows ? L.N : wrows;
     const int64_t a_slab = (int64_t)L.M * Kp;
-    if (!make_map(&maps[0], L.a_hi, Kp, L.M, a_slabs, a_box, a_slab) ||
-        !make_map(&maps[1], L.a_lo, Kp, L.M, a_slabs, a_box, a_slab) ||
-        !make_map(&maps[2], L.w_hi, Kp, L.N, nbr, w_box, L.w_slab) ||
-        !make_map(&maps[3], L.w_lo, Kp, L.N, nbr, w_box, L.w_slab))
-        return cudaErrorInvalidValue;
+    const CUtensorMap* maps[4] = {cached_map(ts, L.a_hi, Kp, L.M, a_slabs, a_box, a_slab),
+                                  cached_map(ts, L.a_lo, Kp, L.M, a_slabs, a_box, a_slab),
+                                  cached_map(ts, L.w_hi, Kp, L.N, nbr, w_box, L.w_slab),
+                                  cached_map(ts, L.w_lo, Kp, L.N, nbr, w_box, L.w_slab)};
+    if (!maps[0] || !maps[1] || !maps[2] || !maps[3]) return cudaErrorInvalidValue;
     TcArgs a;
     a.bias[0] = L.bias[0];
     a.bias[1] = L.bias[1];
@@ -1104,7 +1187,7 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     a.group_n = ctx->sm_count / a.tiles_m;
     if (a.group_n < 1) a.group_n = 1;
     if (a.group_n > a.tiles_n) a.group_n = a.tiles_n;
-    if (const char* e = std::getenv("SAMA_TC_GROUP")) { const int g = std::atoi(e); if (g >= 1 && g <= a.tiles_n) a.group_n = g; }
+    if (ts->group >= 1 && ts->group <= a.tiles_n) a.group_n = ts->group;
     const int items = a.tiles_m * a.tiles_n * nbr;
     const int sms = ctx->sm_count;
     KernelScope scope(ctx, SAMA_K_GEMM_TF32X3, L.layer, st);
@@ -1112,10 +1195,12 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     // its small kernels (the direct gradient, see run_meta_grad_tc).
     PdlScope pdl(pdl_enabled() ? 1 : 0);
     // eight epilogue warps (two per lane quarter, each taking half of the columns) except on the 16-wide tile
-    if (pair) return launch_tc<256, true, 8>(maps, a, items, sms, st, ctx->tc_ws_floats, ctx->tc_flags ? kTcFlags : 0);
-    if (bn == 16) return launch_tc<16, false, 4>(maps, a, items, sms, st);
-    if (bn == 64) return launch_tc<64, false, 8>(maps, a, items, sms, st);
-    return launch_tc<128, false, 8>(maps, a, items, sms, st);
+    if (pair)
+        return launch_tc<256, true, 8>(maps, a, items, ts->pair_units, !ts->no_tail, st, ctx->tc_ws_floats,
+                                       ctx->tc_flags ? kTcFlags : 0);
+    if (bn == 16) return launch_tc<16, false, 4>(maps, a, items, sms, false, st);
+    if (bn == 64) return launch_tc<64, false, 8>(maps, a, items, sms, false, st);
+    return launch_tc<128, false, 8>(maps, a, items, sms, false, st);
 }
 
 }  // namespace sama

@@ -27,7 +27,8 @@ head_ce_fd_kernel(const float* __restrict__ hp, const float* __restrict__ hm, in
                   const float* __restrict__ bp, const float* __restrict__ bm,
                   const int32_t* __restrict__ y, const float* __restrict__ lambda, int B, int C, int K,
                   const float* __restrict__ eps_fd, float* __restrict__ metagrad,
-                  float* __restrict__ loss_plus, float* __restrict__ loss_minus, DeviceScalars* sc) {
+                  float* __restrict__ loss_plus, float* __restrict__ loss_minus, float* __restrict__ loss_diff,
+                  DeviceScalars* sc) {
     pdl_trigger();
     pdl_wait();
     constexpr int SPB = kWarps / WPS;  // samples per block
@@ -121,9 +122,10 @@ head_ce_fd_kernel(const float* __restrict__ hp, const float* __restrict__ hm, in
     if (loss_plus) loss_plus[i] = lse_p - zyp;
     if (loss_minus) loss_minus[i] = lse_m - zym;
     const float eps = *eps_fd;
+    const float d = (lse_p - lse_m) - (zyp - zym);
+    if (loss_diff) loss_diff[i] = ok ? d : 0.f;   // loss+ - loss- without the rounding of the two losses to fp32
     float out = 0.f;
     if (ok && eps > 0.f) {
-        const float d = (lse_p - lse_m) - (zyp - zym);
         const float sg = 1.0f / (1.0f + expf(-lambda[i]));
         out = -(sg * (1.0f - sg)) * d / (2.0f * eps * (float)B);
     }
@@ -139,7 +141,8 @@ bool head_applicable(int C) { return C >= 1 && C <= 16; }
 cudaError_t launch_head_ce_fd(sama_ctx* ctx, const float* h_plus, const float* h_minus, int ldh,
                               const float* w_plus, const float* w_minus, const float* b_plus, const float* b_minus,
                               const int32_t* y, const float* lambda, int B, int C, int K, const float* eps_fd,
-                              float* metagrad, float* loss_plus, float* loss_minus, cudaStream_t st) {
+                              float* metagrad, float* loss_plus, float* loss_minus, float* loss_diff,
+                              cudaStream_t st) {
     const bool vec = (K % 4 == 0) && (ldh % 4 == 0) && aligned16(h_plus) && aligned16(h_minus) &&
                      aligned16(w_plus) && aligned16(w_minus);
     // a whole block per sample while that still gives every SM a few blocks; a warp per sample beyond
@@ -154,7 +157,7 @@ cudaError_t launch_head_ce_fd(sama_ctx* ctx, const float* h_plus, const float* h
 #define SAMA_HEAD2(CT, V, W)                                                                                       \
     err = launch_dependent(head_ce_fd_kernel<CT, V, W>, dim3(grid), dim3(kWarps * 32), 0, st, h_plus, h_minus, ldh, \
                            w_plus, w_minus, b_plus, b_minus, y, lambda, B, C, K, eps_fd, metagrad, loss_plus,      \
-                           loss_minus, ctx->scalars)
+                           loss_minus, loss_diff, ctx->scalars)
 #define SAMA_HEAD(CT, V) do { if (wps == 4) SAMA_HEAD2(CT, V, 4); else if (wps == 2) SAMA_HEAD2(CT, V, 2); else SAMA_HEAD2(CT, V, 1); } while (0)
     if (C <= 4) { if (vec) SAMA_HEAD(4, true); else SAMA_HEAD(4, false); }
     else if (C <= 10) { if (vec) SAMA_HEAD(10, true); else SAMA_HEAD(10, false); }

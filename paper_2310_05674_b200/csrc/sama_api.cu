@@ -108,8 +108,9 @@ int check_mlp(const sama_mlp_t* mlp) {
 }
 
 int validate_perturb(sama_ctx* ctx, int64_t n, const float* theta, const float* p, const double* p_sumsq,
-                     float alpha, float* theta_plus, float* theta_minus, float* eps_fd_out) {
-    if (!ctx || !theta || !p || !theta_plus || !theta_minus) return SAMA_ERR_NULL;
+                     float alpha, float* theta_plus, float* theta_minus, float* eps_fd_out,
+                     bool outputs_optional = false) {
+    if (!ctx || !theta || !p || (!outputs_optional && (!theta_plus || !theta_minus))) return SAMA_ERR_NULL;
     if (n < 0 || n > ctx->max_n) return SAMA_ERR_SIZE;
     if (!std::isfinite(alpha) || !(alpha > 0.f)) return SAMA_ERR_PARAM;
     if (!aligned(theta, 4) || !aligned(p, 4) || !aligned(theta_plus, 4) || !aligned(theta_minus, 4) ||
@@ -169,10 +170,20 @@ SplitLayout make_split_layout(const sama_mlp_t* mlp) {
         lay.w_off[l] = off;
         lay.w_cnt[l] = (int64_t)din * dout;
         lay.s_off[l] = soff;
+        lay.N[l] = dout;
         off += (int64_t)din * dout + dout;
         soff += (int64_t)dout * lay.Kp[l];
     }
     lay.slab = soff;
+    const int last = mlp->n_layers - 1;
+    lay.head_layer = head_applicable(mlp->dims[last + 1]) ? last : -1;
+    lay.head_cnt = lay.head_layer >= 0 ? lay.w_cnt[last] : 0;
+    int64_t boff = lay.head_cnt;
+    for (int l = 0; l < mlp->n_layers; ++l) {
+        lay.b_off[l] = boff;
+        boff += lay.N[l];
+    }
+    lay.small = (boff + 3) & ~(int64_t)3;
     return lay;
 }
 
@@ -185,7 +196,8 @@ bool tc_fits(const sama_ctx* ctx, const sama_mlp_t* mlp, int32_t B) {
     auto r32 = [](int x) { return (size_t)((x + 31) & ~31); };
     const int L = mlp->n_layers;
     if (ctx->x_split_half == 0 || (size_t)B * r32(mlp->dims[0]) > ctx->x_split_half) return false;
-    if (2 * (size_t)make_split_layout(mlp).slab > ctx->w_split_half) return false;
+    const SplitLayout lay = make_split_layout(mlp);
+    if (2 * (size_t)lay.slab > ctx->w_split_half || (size_t)lay.small > ctx->pm_small_half) return false;
     for (int l = 0; l + 1 < L; ++l)
         if (2 * (size_t)B * r32(mlp->dims[l + 1]) > ctx->a_split_half) return false;
     return true;
@@ -229,8 +241,9 @@ int run_forward_tc(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus
         t.w_hi = w_hi + lay.s_off[l];
         t.w_lo = w_lo + lay.s_off[l];
         t.w_slab = lay.slab;
-        t.bias[0] = theta_plus + lay.w_off[l] + lay.w_cnt[l];
-        t.bias[1] = theta_minus + lay.w_off[l] + lay.w_cnt[l];
+        // biases: from the compact slab the fused perturbation sweep filled, else straight from theta+-
+        t.bias[0] = w_presplit ? ctx->pm_small + lay.b_off[l] : theta_plus + lay.w_off[l] + lay.w_cnt[l];
+        t.bias[1] = w_presplit ? ctx->pm_small + lay.small + lay.b_off[l] : theta_minus + lay.w_off[l] + lay.w_cnt[l];
         t.out_f32[0] = f32_out;
         t.out_f32[1] = f32_out + (int64_t)B * dout;
         t.out_hi = last ? nullptr : ctx->a_split[l & 1];
@@ -258,8 +271,10 @@ int run_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const 
     const bool fits = tc_fits(ctx, mlp, B);
     if (ctx->gemm_mode == 2 && !fits) return SAMA_ERR_SIZE;
     const bool use_tc = ctx->gemm_mode != 1 && fits;
+    ctx->last_forward_path = use_tc ? 2 : 1;
     const bool fused_head = head_applicable(C);
     const float* eps = eps_fd ? eps_fd : &ctx->scalars->eps_fd;
+    float* diff_out = ctx->rw_buf ? ctx->rw_buf + 4 * (size_t)ctx->max_batch : nullptr;
     const int n_gemm = fused_head ? L - 1 : L;  // layers computed as matrix products
     const float* in[2] = {X, X};                // fp32 input of the next stage
     int ld_in = mlp->dims[0];
@@ -307,12 +322,23 @@ int run_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const 
         int64_t off = 0;
         for (int l = 0; l + 1 < L; ++l) off += (int64_t)mlp->dims[l] * mlp->dims[l + 1] + mlp->dims[l + 1];
         const int K = mlp->dims[L - 1];
-        SAMA_CUDA(ctx, launch_head_ce_fd(ctx, in[0], in[1], ld_in, theta_plus + off, theta_minus + off,
-                                         theta_plus + off + (int64_t)K * C, theta_minus + off + (int64_t)K * C, y,
-                                         lambda, B, C, K, eps, metagrad_out, loss_plus_out, loss_minus_out, st));
+        // the head's fp32 weights and biases: from the compact slab after a fused perturbation sweep, else from theta+-
+        const float* wp = theta_plus + off;
+        const float* wm = theta_minus + off;
+        const float* bp = wp + (int64_t)K * C;
+        const float* bm = wm + (int64_t)K * C;
+        if (use_tc && w_presplit) {
+            const SplitLayout lay = make_split_layout(mlp);
+            wp = ctx->pm_small;
+            wm = ctx->pm_small + lay.small;
+            bp = wp + lay.b_off[L - 1];
+            bm = wm + lay.b_off[L - 1];
+        }
+        SAMA_CUDA(ctx, launch_head_ce_fd(ctx, in[0], in[1], ld_in, wp, wm, bp, bm, y,
+                                         lambda, B, C, K, eps, metagrad_out, loss_plus_out, loss_minus_out, diff_out, st));
     } else {
         SAMA_CUDA(ctx, launch_ce_fd(ctx, in[0], in[1], C, y, lambda, B, C, eps, metagrad_out, loss_plus_out,
-                                    loss_minus_out, st));
+                                    loss_minus_out, diff_out, st));
     }
     return SAMA_OK;
 }
@@ -364,7 +390,7 @@ int sama_create(sama_ctx** out, int device, int64_t max_n, int32_t max_batch, co
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return SAMA_ERR_CUDA; }
     ctx->sm_count = prop.multiProcessorCount;
-    if (const char* t = std::getenv("SAMA_TC_TILE")) ctx->tile_override = std::atoi(t);
+    if (const char* e = std::getenv("SAMA_NO_FUSED_SWEEP")) ctx->no_fused_sweep = (e[0] == '1');
     bool ok = cudaMalloc(&ctx->scalars, sizeof(DeviceScalars)) == cudaSuccess &&
               cudaMemset(ctx->scalars, 0, sizeof(DeviceScalars)) == cudaSuccess &&
               cudaMalloc(&ctx->partials, sizeof(double) * kMaxPartials) == cudaSuccess;
@@ -391,6 +417,8 @@ int sama_create(sama_ctx** out, int device, int64_t max_n, int32_t max_batch, co
         ctx->a_split_half = 2 * (size_t)max_batch * amax;
         ok = ok && cudaMalloc(&ctx->x_split, sizeof(float) * 2 * ctx->x_split_half) == cudaSuccess &&
              cudaMalloc(&ctx->w_split, sizeof(float) * 2 * ctx->w_split_half) == cudaSuccess;
+        ctx->pm_small_half = (size_t)make_split_layout(mlp).small;
+        ok = ok && cudaMalloc(&ctx->pm_small, sizeof(float) * 2 * ctx->pm_small_half) == cudaSuccess;
         ctx->tc_ws_floats = (size_t)ctx->sm_count * 128 * 256;
         ok = ok && cudaMalloc(&ctx->tc_ws, sizeof(float) * ctx->tc_ws_floats) == cudaSuccess &&
              cudaMalloc(&ctx->tc_flags, sizeof(int) * kTcFlags) == cudaSuccess &&
@@ -402,6 +430,19 @@ int sama_create(sama_ctx** out, int device, int64_t max_n, int32_t max_batch, co
         if (ok && amax > 0)
             ok = cudaMalloc(&ctx->a_split[0], sizeof(float) * 2 * ctx->a_split_half) == cudaSuccess &&
                  cudaMalloc(&ctx->a_split[1], sizeof(float) * 2 * ctx->a_split_half) == cudaSuccess;
+        ok = ok && cudaMalloc(&ctx->rw_partials, sizeof(double) * (size_t)kMaxReweightBlocks *
+                                                     (3 * kMaxReweightHidden + 1)) == cudaSuccess &&
+             cudaMalloc(&ctx->rw_buf, sizeof(float) * 5 * (size_t)max_batch) == cudaSuccess &&
+             cudaMemset(ctx->rw_buf, 0, sizeof(float) * 5 * (size_t)max_batch) == cudaSuccess;
+        if (ok) {
+            const cudaError_t e = tc_state_create(ctx);
+            if (e != cudaSuccess) {
+                ctx->last_cuda_error = (int)e;
+                cudaGetLastError();
+                sama_destroy(ctx);
+                return SAMA_ERR_CUDA;
+            }
+        }
     }
     if (!ok || cudaDeviceSynchronize() != cudaSuccess) {
         cudaGetLastError();
@@ -429,6 +470,12 @@ int sama_destroy(sama_ctx* ctx) {
     cudaFree(ctx->mg_ws);
     cudaFree(ctx->mg_tc);
     cudaFree(ctx->stage);
+    cudaFree(ctx->pm_small);
+    cudaFree(ctx->pm_scratch);
+    cudaFree(ctx->rw_partials);
+    cudaFree(ctx->rw_buf);
+    cudaFree(ctx->br_partials);
+    tc_state_destroy(ctx);
     if (ctx->prof) {
         for (auto& r : ctx->prof->records) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
         delete ctx->prof;
@@ -489,10 +536,11 @@ int sama_step(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* thet
     AdaptConsts c;
     rc = validate_adapt(ctx->max_n, n, m, s, g_base, g_meta, adam, p_out, nullptr, &c);
     if (rc != SAMA_OK) return rc;
-    rc = validate_perturb(ctx, n, theta, p_out, nullptr, alpha, theta_plus, theta_minus, nullptr);
+    rc = validate_perturb(ctx, n, theta, p_out, nullptr, alpha, theta_plus, theta_minus, nullptr, true);
     if (rc != SAMA_OK) return rc;
-    rc = validate_fd(ctx, mlp, theta_plus, theta_minus, X, y, lambda, B, nullptr, metagrad_out, loss_plus_out,
-                     loss_minus_out);
+    // (theta+- are optional here; the forward's own checks get stand-ins that overlap nothing)
+    rc = validate_fd(ctx, mlp, theta_plus ? theta_plus : theta, theta_minus ? theta_minus : theta, X, y, lambda, B,
+                     nullptr, metagrad_out, loss_plus_out, loss_minus_out);
     if (rc != SAMA_OK) return rc;
     // outputs of the early stages must not be inputs of the later ones
     const size_t nb = (size_t)n * 4, bb = (size_t)B * 4;
@@ -514,11 +562,15 @@ int sama_step(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* thet
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return SAMA_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;
-    SAMA_CUDA(ctx, launch_adapt_sumsq(ctx, n, m, s, c.identity ? nullptr : g_base, g_meta, c, p_out, nullptr, st));
     // With the tensor-core forward, the perturbation sweep also emits the TF32 operand split of W+-.
     const SplitLayout lay = make_split_layout(mlp);
     const bool fused = ctx->gemm_mode != 1 && tc_fits(ctx, mlp, B) &&
                        perturb_split_applicable(lay, theta, p_out, theta_plus, theta_minus);
+    // ... and for a model small enough, adaptation and norm join it in one launch
+    const bool one_launch = fused && aligned(g_meta, 16) && (c.identity || (aligned(m, 16) && aligned(s, 16))) &&
+                            (c.identity || !g_base || aligned(g_base, 16)) && fused_sweep_applicable(ctx, n);
+    if (!one_launch)
+        SAMA_CUDA(ctx, launch_adapt_sumsq(ctx, n, m, s, c.identity ? nullptr : g_base, g_meta, c, p_out, nullptr, st));
     // ... and, where the batch allows vector access, the split of X as well (one launch fewer)
     XSplitJob xjob;
     std::memset(&xjob, 0, sizeof(xjob));
@@ -532,15 +584,149 @@ int sama_step(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* thet
         xjob.cols = mlp->dims[0];
         xjob.ld_out = (mlp->dims[0] + 31) & ~31;
     }
-    if (fused)
+    if (one_launch) {
+        SAMA_CUDA(ctx, launch_fused_sweep(ctx, n, theta, m, s, c.identity ? nullptr : g_base, g_meta, c, alpha, p_out,
+                                          theta_plus, theta_minus, lay, ctx->w_split, ctx->w_split + ctx->w_split_half,
+                                          ctx->pm_small, xjob, st));
+    } else if (fused) {
         SAMA_CUDA(ctx, launch_perturb_split(ctx, n, theta, p_out, &ctx->scalars->sumsq, alpha, theta_plus,
                                             theta_minus, nullptr, lay, ctx->w_split,
-                                            ctx->w_split + ctx->w_split_half, xjob, st));
-    else
+                                            ctx->w_split + ctx->w_split_half, ctx->pm_small, xjob, st));
+    } else {
+        // this path's forward reads theta+- themselves: a caller that wants neither gets them in scratch
+        if (!theta_plus || !theta_minus) {
+            const size_t nn = ((size_t)n + 63) & ~(size_t)63;
+            if (ctx->pm_scratch_floats < 2 * nn) {
+                SAMA_CUDA(ctx, cudaStreamSynchronize(st));
+                cudaFree(ctx->pm_scratch);
+                ctx->pm_scratch = nullptr;
+                ctx->pm_scratch_floats = 0;
+                if (cudaMalloc(&ctx->pm_scratch, sizeof(float) * 2 * nn) != cudaSuccess) { cudaGetLastError(); return SAMA_ERR_NOMEM; }
+                ctx->pm_scratch_floats = 2 * nn;
+            }
+            if (!theta_plus) theta_plus = ctx->pm_scratch;
+            if (!theta_minus) theta_minus = ctx->pm_scratch + nn;
+        }
         SAMA_CUDA(ctx, launch_perturb(ctx, n, theta, p_out, &ctx->scalars->sumsq, alpha, theta_plus, theta_minus,
                                       nullptr, st));
+    }
     return run_fd(ctx, mlp, theta_plus, theta_minus, X, y, lambda, B, nullptr, metagrad_out, loss_plus_out,
                   loss_minus_out, st, fused, x_fused);
+}
+
+int sama_fd_metagrad_reweight(sama_ctx* ctx, int32_t B, const float* loss_plus, const float* loss_minus,
+                              const float* loss_diff, int32_t hidden, const float* lambda_r, const float* eps_fd,
+                              int32_t B_norm, float* metagrad_r_out, void* stream) {
+    if (!ctx || !loss_minus || (!loss_plus && !loss_diff) || !lambda_r || !metagrad_r_out) return SAMA_ERR_NULL;
+    if (!ctx->rw_partials || B < 1 || B > ctx->max_batch || B_norm < 1 || hidden < 1 || hidden > kMaxReweightHidden)
+        return SAMA_ERR_SIZE;
+    if (!aligned(loss_plus, 4) || !aligned(loss_minus, 4) || !aligned(loss_diff, 4) || !aligned(lambda_r, 4) ||
+        !aligned(eps_fd, 4) || !aligned(metagrad_r_out, 4))
+        return SAMA_ERR_ALIGN;
+    const size_t bb = (size_t)B * 4, lb = (size_t)(3 * hidden + 1) * 4;
+    if (overlaps(metagrad_r_out, lb, loss_plus, bb) || overlaps(metagrad_r_out, lb, loss_minus, bb) ||
+        overlaps(metagrad_r_out, lb, loss_diff, bb) ||
+        overlaps(metagrad_r_out, lb, lambda_r, lb) || overlaps(metagrad_r_out, lb, eps_fd, 4))
+        return SAMA_ERR_OVERLAP;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SAMA_ERR_CUDA;
+    SAMA_CUDA(ctx, launch_reweight_fd(ctx, loss_plus, loss_minus, loss_diff, B, B_norm, hidden, lambda_r,
+                                      eps_fd ? eps_fd : &ctx->scalars->eps_fd, metagrad_r_out, (cudaStream_t)stream));
+    return SAMA_OK;
+}
+
+int sama_step_reweight(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* theta, const float* m,
+                       const float* s, const float* g_base, const float* g_meta, const sama_adam_t* adam,
+                       float alpha, const float* X, const int32_t* y, int32_t B, int32_t hidden,
+                       const float* lambda_r, float* p_out, float* theta_plus, float* theta_minus,
+                       float* metagrad_r_out, float* loss_plus_out, float* loss_minus_out, void* stream) {
+    if (!ctx || !lambda_r || !metagrad_r_out) return SAMA_ERR_NULL;
+    if (!ctx->rw_buf || B < 1 || B > ctx->max_batch || hidden < 1 || hidden > kMaxReweightHidden) return SAMA_ERR_SIZE;
+    if (!aligned(lambda_r, 4) || !aligned(metagrad_r_out, 4)) return SAMA_ERR_ALIGN;
+    const size_t nb = (size_t)(n > 0 ? n : 0) * 4, lb = (size_t)(3 * hidden + 1) * 4;
+    if (overlaps(metagrad_r_out, lb, p_out, nb) || overlaps(metagrad_r_out, lb, theta_plus, nb) ||
+        overlaps(metagrad_r_out, lb, theta_minus, nb) || overlaps(metagrad_r_out, lb, lambda_r, lb) ||
+        overlaps(metagrad_r_out, lb, loss_plus_out, (size_t)B * 4) || overlaps(metagrad_r_out, lb, loss_minus_out, (size_t)B * 4) ||
+        overlaps(lambda_r, lb, p_out, nb) || overlaps(lambda_r, lb, theta_plus, nb) || overlaps(lambda_r, lb, theta_minus, nb))
+        return SAMA_ERR_OVERLAP;
+    // the forward pass and its per-sample losses are those of sama_step; the per-sample logits it wants are the
+    // context's zeros and its per-sample meta gradient goes to scratch
+    float* lp = loss_plus_out ? loss_plus_out : ctx->rw_buf;
+    float* lm = loss_minus_out ? loss_minus_out : ctx->rw_buf + ctx->max_batch;
+    const float* zeros = ctx->rw_buf + 2 * (size_t)ctx->max_batch;
+    float* scratch = ctx->rw_buf + 3 * (size_t)ctx->max_batch;
+    const int rc = sama_step(ctx, mlp, n, theta, m, s, g_base, g_meta, adam, alpha, X, y, zeros, B, p_out, theta_plus,
+                             theta_minus, scratch, lp, lm, stream);
+    if (rc != SAMA_OK) return rc;
+    return sama_fd_metagrad_reweight(ctx, B, lp, lm, ctx->rw_buf + 4 * (size_t)ctx->max_batch, hidden, lambda_r, nullptr, B,
+                                     metagrad_r_out, stream);
+}
+
+int sama_biasreg_direct_grad(sama_ctx* ctx, int32_t d, int32_t n_val, const float* Xv, const float* yv,
+                             const float* w, float* g_meta_out, float* meta_loss_out, void* stream) {
+    if (!ctx || !Xv || !yv || !w || !g_meta_out) return SAMA_ERR_NULL;
+    if (d < 1 || n_val < 1 || d > 24 * 1024 || (int64_t)d > ctx->max_n) return SAMA_ERR_SIZE;
+    if (!aligned(Xv, 4) || !aligned(yv, 4) || !aligned(w, 4) || !aligned(g_meta_out, 4) || !aligned(meta_loss_out, 4))
+        return SAMA_ERR_ALIGN;
+    const size_t db = (size_t)d * 4;
+    if (overlaps(g_meta_out, db, Xv, (size_t)n_val * d * 4) || overlaps(g_meta_out, db, yv, (size_t)n_val * 4) ||
+        overlaps(g_meta_out, db, w, db) || overlaps(g_meta_out, db, meta_loss_out, 4))
+        return SAMA_ERR_OVERLAP;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SAMA_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t need = (size_t)biasreg_grid(ctx, n_val) * ((size_t)d + 1);
+    if (ctx->br_partials_doubles < need) {
+        SAMA_CUDA(ctx, cudaStreamSynchronize(st));
+        cudaFree(ctx->br_partials);
+        ctx->br_partials = nullptr;
+        ctx->br_partials_doubles = 0;
+        const size_t take = (size_t)ctx->sm_count * ((size_t)d + 1);
+        if (cudaMalloc(&ctx->br_partials, sizeof(double) * take) != cudaSuccess) { cudaGetLastError(); return SAMA_ERR_NOMEM; }
+        ctx->br_partials_doubles = take;
+    }
+    SAMA_CUDA(ctx, launch_biasreg_direct_grad(ctx, d, n_val, Xv, yv, w, g_meta_out, meta_loss_out, st));
+    return SAMA_OK;
+}
+
+int sama_biasreg_fd_metagrad(sama_ctx* ctx, int64_t d, const float* w_plus, const float* w_minus,
+                             const float* lambda, float beta, const float* eps_fd, float* metagrad_out,
+                             void* stream) {
+    if (!ctx || !w_plus || !w_minus || !lambda || !metagrad_out) return SAMA_ERR_NULL;
+    if (d < 0 || d > ctx->max_n) return SAMA_ERR_SIZE;
+    if (!std::isfinite(beta) || !(beta >= 0.f)) return SAMA_ERR_PARAM;
+    if (!aligned(w_plus, 4) || !aligned(w_minus, 4) || !aligned(lambda, 4) || !aligned(eps_fd, 4) ||
+        !aligned(metagrad_out, 4))
+        return SAMA_ERR_ALIGN;
+    const size_t db = (size_t)d * 4;
+    if (overlaps(metagrad_out, db, w_plus, db) || overlaps(metagrad_out, db, w_minus, db) ||
+        overlaps(metagrad_out, db, lambda, db) || overlaps(metagrad_out, db, eps_fd, 4))
+        return SAMA_ERR_OVERLAP;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SAMA_ERR_CUDA;
+    SAMA_CUDA(ctx, launch_biasreg_fd(ctx, d, w_plus, w_minus, lambda, beta, eps_fd ? eps_fd : &ctx->scalars->eps_fd,
+                                     metagrad_out, (cudaStream_t)stream));
+    return SAMA_OK;
+}
+
+int sama_biasreg_step(sama_ctx* ctx, int32_t d, int32_t n_val, const float* Xv, const float* yv, const float* w,
+                      const float* lambda, float beta, const float* m, const float* s, const float* g_base,
+                      const sama_adam_t* adam, float alpha, float* g_meta_out, float* p_out, float* w_plus,
+                      float* w_minus, float* metagrad_out, void* stream) {
+    if (!ctx || !lambda || !metagrad_out || !p_out || !w_plus || !w_minus || !adam) return SAMA_ERR_NULL;
+    // the four stages validate their own arguments; what only the chain can get wrong is checked here
+    const size_t db = (size_t)(d > 0 ? d : 0) * 4;
+    if (overlaps(metagrad_out, db, p_out, db) || overlaps(metagrad_out, db, g_meta_out, db) ||
+        overlaps(w_plus, db, g_meta_out, db) || overlaps(w_minus, db, g_meta_out, db) ||
+        overlaps(p_out, db, lambda, db) || overlaps(w_plus, db, lambda, db) || overlaps(w_minus, db, lambda, db))
+        return SAMA_ERR_OVERLAP;
+    int rc = sama_biasreg_direct_grad(ctx, d, n_val, Xv, yv, w, g_meta_out, nullptr, stream);
+    if (rc != SAMA_OK) return rc;
+    rc = sama_adapt(ctx, d, m, s, g_base, g_meta_out, adam, p_out, nullptr, stream);
+    if (rc != SAMA_OK) return rc;
+    rc = sama_perturb(ctx, d, w, p_out, &ctx->scalars->sumsq, alpha, w_plus, w_minus, nullptr, stream);
+    if (rc != SAMA_OK) return rc;
+    return sama_biasreg_fd_metagrad(ctx, d, w_plus, w_minus, lambda, beta, nullptr, metagrad_out, stream);
 }
 
 int sama_meta_grad(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta, const float* X_meta,
@@ -578,11 +764,11 @@ int sama_step_host(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float*
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return SAMA_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;
-    // staging layout (floats): theta m s g_base g_meta p theta+ theta- | X | lambda | metagrad | y
+    // staging layout (floats): theta m s g_base g_meta p theta- | X | lambda | metagrad | y
     const size_t nn = ((size_t)n + 63) & ~(size_t)63;
     const size_t xs = (((size_t)B * mlp->dims[0]) + 63) & ~(size_t)63;
     const size_t bs = ((size_t)B + 63) & ~(size_t)63;
-    const size_t need = (8 * nn + xs + 3 * bs) * sizeof(float);
+    const size_t need = (7 * nn + xs + 3 * bs) * sizeof(float);
     if (ctx->stage_bytes < need) {
         SAMA_CUDA(ctx, cudaStreamSynchronize(st));
         cudaFree(ctx->stage);
@@ -597,8 +783,7 @@ int sama_step_host(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float*
     float* d_g = d_s + nn;
     float* d_gm = d_g + nn;
     float* d_p = d_gm + nn;
-    float* d_tp = d_p + nn;
-    float* d_tm = d_tp + nn;
+    float* d_tm = d_p + nn;
     float* d_X = d_tm + nn;
     float* d_lam = d_X + xs;
     float* d_mg = d_lam + bs;
@@ -613,8 +798,8 @@ int sama_step_host(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float*
     SAMA_CUDA(ctx, cudaMemcpyAsync(d_y, y_host, (size_t)B * 4, cudaMemcpyHostToDevice, st));
     SAMA_CUDA(ctx, cudaMemcpyAsync(d_lam, lambda_host, (size_t)B * 4, cudaMemcpyHostToDevice, st));
     rc = sama_step(ctx, mlp, n, d_theta, m_host ? d_m : nullptr, s_host ? d_s : nullptr,
-                   g_base_host ? d_g : nullptr, d_gm, adam, alpha, d_X, d_y, d_lam, B, d_p, d_tp, d_tm, d_mg,
-                   nullptr, nullptr, stream);
+                   g_base_host ? d_g : nullptr, d_gm, adam, alpha, d_X, d_y, d_lam, B, d_p, nullptr,
+                   theta_minus_out_host ? d_tm : nullptr, d_mg, nullptr, nullptr, stream);
     if (rc != SAMA_OK) return rc;
     SAMA_CUDA(ctx, cudaMemcpyAsync(metagrad_out_host, d_mg, (size_t)B * 4, cudaMemcpyDeviceToHost, st));
     if (eps_fd_out_host)
@@ -626,6 +811,7 @@ int sama_step_host(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float*
 }
 
 double* sama_ctx_sumsq(sama_ctx* ctx) { return ctx ? &ctx->scalars->sumsq : nullptr; }
+float* sama_ctx_loss_diff(sama_ctx* ctx) { return (ctx && ctx->rw_buf) ? ctx->rw_buf + 4 * (size_t)ctx->max_batch : nullptr; }
 float* sama_ctx_eps_fd(sama_ctx* ctx) { return ctx ? &ctx->scalars->eps_fd : nullptr; }
 
 int sama_device_status(sama_ctx* ctx, void* stream, int32_t* status_out) {
@@ -652,6 +838,8 @@ int sama_set_gemm_mode(sama_ctx* ctx, int mode) {
 
 int64_t sama_launch_count(sama_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+int sama_last_forward_path(sama_ctx* ctx) { return ctx ? ctx->last_forward_path : 0; }
+
 int sama_profile_enable(sama_ctx* ctx, int32_t on) {
     if (!ctx) return SAMA_ERR_NULL;
     DeviceGuard guard(ctx->device);
@@ -663,6 +851,7 @@ int sama_profile_enable(sama_ctx* ctx, int32_t on) {
     for (auto& r : ctx->prof->records) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
     ctx->prof->records.clear();
     ctx->prof->on = (on != 0);
+    ctx->prof->grouped = (on == 2);
     return SAMA_OK;
 }
 
@@ -680,7 +869,7 @@ int sama_profile_collect(sama_ctx* ctx, sama_kernel_time_t* out, int32_t capacit
         cudaEventDestroy(r.start);
         cudaEventDestroy(r.stop);
         if (e != cudaSuccess) { ctx->prof->records.clear(); return cuda_fail(ctx, e); }
-        if (k < capacity) { out[k].kind = r.kind; out[k].layer = r.layer; out[k].ms = ms; ++k; }
+        if (k < capacity) { out[k].kind = r.kind; out[k].layer = r.layer; out[k].ms = ms; out[k].launches = r.launches; ++k; }
     }
     ctx->prof->records.clear();
     *count_out = k;

@@ -12,14 +12,16 @@ namespace sama {
 constexpr int kMaxLayers = 16;
 constexpr int kMaxPartials = 4096;  // upper bound on the grid of the reduction kernels
 constexpr int kTcFlags = 1024;      // arrival counters of the tensor-core kernel's shared tail tiles
+constexpr int kMaxReweightHidden = 256;  // widest hidden layer of the shared reweighting network
+constexpr int kMaxReweightBlocks = 512;  // upper bound on the grid of its reduction
 
 // Device scalars owned by a context.
 struct DeviceScalars {
     double sumsq;          // sum p^2 of the last adapt
     float eps_fd;          // alpha / ||p|| of the last perturb
     int32_t status;        // OR of SAMA_DEV_* bits
-    unsigned int counter;  // arrival counter of the last-block-done reduction (returns to 0)
-    unsigned int pad;
+    unsigned int counter;  // arrival counter of the last-block-done reductions and of the fused sweep's grid barrier (returns to 0)
+    unsigned int departed; // blocks that have left the fused sweep's grid barrier (returns to 0)
 };
 
 // Host-precomputed constants of the Adam adaptation matrix (Appendix C).
@@ -43,6 +45,14 @@ struct SplitLayout {
     int64_t w_cnt[kMaxLayers];  // d_l * d_{l-1}
     int64_t s_off[kMaxLayers];  // offset of layer l inside a slab
     int64_t slab;               // floats per slab = sum_l d_l * Kp_l
+    // What the forward pass reads in fp32 besides the split operands, kept compact per branch ("small slab"):
+    // the weights of a narrow last layer that the fused head kernel multiplies itself (first, so that every
+    // block starts at a multiple of 4), then every layer's bias.
+    int32_t N[kMaxLayers];      // d_l (length of layer l's bias)
+    int64_t b_off[kMaxLayers];  // offset of layer l's bias inside a small slab
+    int head_layer;             // index of the layer whose fp32 weights are kept (the fused head's), or -1
+    int64_t head_cnt;           // its weight count (at offset 0 of the small slab), else 0
+    int64_t small;              // floats per small slab
 };
 
 // The batch X as an extra job of the fused perturbation sweep: its TF32 hi/lo split, rows padded to ld_out.
@@ -56,11 +66,12 @@ struct XSplitJob {
 };
 
 struct ProfRecord {
-    int kind, layer;
+    int kind, layer, launches;
     cudaEvent_t start, stop;
 };
 struct Profiler {
     bool on = false;
+    bool grouped = false;  // consecutive launches of one kind share a record (one event pair around the run)
     std::vector<ProfRecord> records;
 };
 
@@ -74,8 +85,11 @@ struct sama_ctx {
     int32_t max_width;    // widest hidden layer the forward workspace covers, 0 if none
     int32_t max_classes;  // largest d_L covered, 0 if the context has no forward workspace
     int gemm_mode;        // 0 auto, 1 ffma, 2 3xTF32
-    int tile_override;    // 0, or an N-tile width forced through the SAMA_TC_TILE environment variable (tuning aid)
     int last_cuda_error;
+    int fused_sweep_blocks;  // co-resident blocks per SM of the fused sweep kernel on this device (0: not yet asked, -1: unavailable)
+    int no_fused_sweep;      // SAMA_NO_FUSED_SWEEP=1 (experiment switch, read at sama_create)
+    int last_forward_path;  // how the last forward pass multiplied matrices: 0 none yet, 1 fp32 FMA, 2 tensor cores
+    void* tc_state;       // host: state of the tensor-core path (switches, unit counts, tensor-map cache), or null
     int64_t launches;
     sama::DeviceScalars* scalars;  // device
     double* partials;              // device [kMaxPartials]
@@ -86,6 +100,10 @@ struct sama_ctx {
     float* w_split;                // device [hi, lo][2 branches][slab]: every layer's W, rows padded to 32
     float* a_split[2];             // device, ping-pong: [2][2][max_batch][round32(max hidden)]
     size_t x_split_half, w_split_half, a_split_half;  // floats per hi (or lo) part; 0 = path unavailable
+    float* pm_small;               // device [2 branches][pm_small_half]: fp32 biases and fused-head weights of theta+ / theta-
+    size_t pm_small_half;
+    float* pm_scratch;             // device [2][n]: theta+ / theta- when the caller wants neither and the forward needs them (allocated on first use)
+    size_t pm_scratch_floats;
     float* tc_ws;                  // device: partial tiles of the tensor-core path's K-split (one 128 x 256 tile per SM)
     int* tc_flags;                 // device [kTcFlags], zero between launches
     size_t tc_ws_floats;
@@ -93,6 +111,11 @@ struct sama_ctx {
     size_t mg_ws_floats;
     float* mg_tc;                  // device: TF32 operand buffers of the direct gradient's tensor-core path
     size_t mg_tc_floats;
+    double* rw_partials;           // device [kMaxReweightBlocks][3 kMaxReweightHidden + 1]: block partials of the reweighting-network gradient
+    float* rw_buf;                 // device [5][max_batch]: losses of both branches, zero logits, scratch meta gradient (sama_step_reweight);
+                                   // [4]: loss+ - loss- of the last forward pass, as formed inside its last kernel
+    double* br_partials;           // device: block partials of the biased-regression direct gradient (allocated on first use)
+    size_t br_partials_doubles;
     float* stage;                  // device: staging of the host entry point (allocated on first use)
     size_t stage_bytes;
     sama::Profiler* prof;          // host
@@ -108,11 +131,20 @@ struct KernelScope {
     KernelScope(sama_ctx* c, int kind, int layer, cudaStream_t s) : ctx(c), st(s) {
         ctx->launches += 1;
         if (ctx->prof && ctx->prof->on) {
-            ProfRecord r{kind, layer, nullptr, nullptr};
+            std::vector<ProfRecord>& recs = ctx->prof->records;
+            if (ctx->prof->grouped && !recs.empty() && recs.back().kind == kind) {
+                // same kind as the launch before: no event in between (it would serialise the two launches and
+                // undo their dependent-launch overlap); the record's stop event is recorded again after this one
+                recs.back().launches += 1;
+                recs.back().layer = -1;
+                stop = recs.back().stop;
+                return;
+            }
+            ProfRecord r{kind, layer, 1, nullptr, nullptr};
             if (cudaEventCreate(&r.start) == cudaSuccess && cudaEventCreate(&r.stop) == cudaSuccess) {
                 cudaEventRecord(r.start, st);
                 stop = r.stop;
-                ctx->prof->records.push_back(r);
+                recs.push_back(r);
             }
         }
     }
@@ -182,11 +214,19 @@ cudaError_t launch_sumsq(sama_ctx* ctx, int64_t n, const float* p, cudaStream_t 
 cudaError_t launch_perturb(sama_ctx* ctx, int64_t n, const float* theta, const float* p, const double* sumsq,
                            float alpha, float* theta_plus, float* theta_minus, float* eps_fd_out, cudaStream_t st);
 // perturb that also writes the TF32 hi/lo split of every weight matrix of theta+ and theta- (same sweep)
+// adaptation + norm + perturbation + operand split in ONE cooperative launch, for models small enough that p
+// stays in registers between the two halves (a grid-wide barrier with a bounded wait separates them)
+bool fused_sweep_applicable(sama_ctx* ctx, int64_t n);
+cudaError_t launch_fused_sweep(sama_ctx* ctx, int64_t n, const float* theta, const float* m, const float* s,
+                               const float* g_base, const float* g_meta, const AdaptConsts& c, float alpha, float* p_out,
+                               float* theta_plus, float* theta_minus, const SplitLayout& lay, float* hi, float* lo,
+                               float* small, const XSplitJob& xjob, cudaStream_t st);
 bool perturb_split_applicable(const SplitLayout& lay, const float* theta, const float* p, const float* theta_plus,
                               const float* theta_minus);
 cudaError_t launch_perturb_split(sama_ctx* ctx, int64_t n, const float* theta, const float* p, const double* sumsq,
                                  float alpha, float* theta_plus, float* theta_minus, float* eps_fd_out,
-                                 const SplitLayout& lay, float* hi, float* lo, const XSplitJob& xjob, cudaStream_t st);
+                                 const SplitLayout& lay, float* hi, float* lo, float* small, const XSplitJob& xjob,
+                                 cudaStream_t st);
 
 // One layer of both branches: C[b] = act(A[b] * W[b]^T + bias[b]) for b in {0, 1}
 struct GemmArgs {
@@ -228,18 +268,33 @@ cudaError_t launch_split_transpose_tf32(sama_ctx* ctx, const float* src, int64_t
 cudaError_t launch_split_tf32(sama_ctx* ctx, const float* src0, const float* src1, int branches, int64_t rows,
                               int cols, float* hi, float* lo, int64_t slab, cudaStream_t st);
 cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st);
+cudaError_t tc_state_create(sama_ctx* ctx);  // with ctx->device current and ctx->sm_count set
+void tc_state_destroy(sama_ctx* ctx);
 
 // ce_fd.cu
 cudaError_t launch_ce_fd(sama_ctx* ctx, const float* z_plus, const float* z_minus, int ldz, const int32_t* y,
                          const float* lambda, int B, int C, const float* eps_fd, float* metagrad,
-                         float* loss_plus, float* loss_minus, cudaStream_t st);
+                         float* loss_plus, float* loss_minus, float* loss_diff, cudaStream_t st);
 
 // head_ce_fd.cu : narrow last layer (C <= 16) + cross-entropy + central difference in one kernel
 bool head_applicable(int C);
 cudaError_t launch_head_ce_fd(sama_ctx* ctx, const float* h_plus, const float* h_minus, int ldh,
                               const float* w_plus, const float* w_minus, const float* b_plus, const float* b_minus,
                               const int32_t* y, const float* lambda, int B, int C, int K, const float* eps_fd,
-                              float* metagrad, float* loss_plus, float* loss_minus, cudaStream_t st);
+                              float* metagrad, float* loss_plus, float* loss_minus, float* loss_diff,
+                              cudaStream_t st);
+
+// reweight.cu : Eq. 5 with the shared reweighting network of Sec. 4.1
+cudaError_t launch_reweight_fd(sama_ctx* ctx, const float* loss_plus, const float* loss_minus,
+                               const float* loss_diff, int B, int B_norm, int H, const float* lambda_r,
+                               const float* eps_fd, float* out, cudaStream_t st);
+
+// biasreg.cu : the biased-regression objective of Appendix E
+int biasreg_grid(const sama_ctx* ctx, int n_val);
+cudaError_t launch_biasreg_direct_grad(sama_ctx* ctx, int d, int n_val, const float* Xv, const float* yv,
+                                       const float* w, float* g_out, float* loss_out, cudaStream_t st);
+cudaError_t launch_biasreg_fd(sama_ctx* ctx, int64_t d, const float* w_plus, const float* w_minus,
+                              const float* lambda, float beta, const float* eps_fd, float* out, cudaStream_t st);
 
 // meta_grad.cu : direct gradient dL_meta/dtheta (Eq. 1)
 size_t meta_grad_workspace_floats(const sama_mlp_t* mlp, int64_t B);

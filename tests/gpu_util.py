@@ -66,14 +66,15 @@ def run_adapt(ctx, w, adam, use_gbase=True, inplace=False, shift=0):
     return p.cpu().numpy()[:n], float(ss.item()), p, ss
 
 
-def run_step(ctx, cfg, w, adam, alpha, use_gbase=True, want_losses=True):
+def run_step(ctx, cfg, w, adam, alpha, use_gbase=True, want_losses=True, want_plus=True, want_minus=True):
     n, Bsz = w["theta"].size, cfg.batch
     t = {k: dev(w[k]) for k in ["theta", "m", "s", "g_meta", "X", "y", "lam"]}
     gb = dev(w["g_base"]) if use_gbase else None
-    f = lambda k: torch.empty(k, dtype=torch.float32, device=DEV)
+    f = lambda k: torch.full((k,), float("nan"), dtype=torch.float32, device=DEV)
     p, tp, tm, mg, lp, lm = f(n), f(n), f(n), f(Bsz), f(Bsz), f(Bsz)
     B.sama_step(ctx.h, ctx.mlp, n, t["theta"], t["m"], t["s"], gb, t["g_meta"], adam, alpha, t["X"], t["y"],
-                t["lam"], Bsz, p, tp, tm, mg, lp if want_losses else None, lm if want_losses else None)
+                t["lam"], Bsz, p, tp if want_plus else None, tm if want_minus else None, mg,
+                lp if want_losses else None, lm if want_losses else None)
     torch.cuda.synchronize()
     out = {"p": p.cpu().numpy(), "theta_plus": tp.cpu().numpy(), "theta_minus": tm.cpu().numpy(),
            "metagrad": mg.cpu().numpy(), "loss_plus": lp.cpu().numpy(), "loss_minus": lm.cpu().numpy(),
@@ -154,12 +155,11 @@ def fd_errors(got, ref):
 
 def assert_fd_close(got, ref, what="metagrad", norm_tol=2e-3):
     """FD meta-gradient: |a-b| <= max(2e-3 |b|, 1e-6) elementwise (the stated
-    bar), and a bound on the whole vector in the 2-norm, which is scale-free
-    and so still bites when the 1/B factor pushes every entry under the
-    absolute floor.  The quotient amplifies the fp32 rounding of the two
-    forward passes by 1/(2 eps_fd): at the paper's default alpha = 1 the norm
-    bound is the same 2e-3; at alpha = 1e-2 the rounding is 100x larger
-    relative to the signal and callers pass 2e-2."""
+    bar), and the same relative 2e-3 on the whole vector in the 2-norm, which is
+    scale-free and so still bites when the 1/B factor pushes every entry under
+    the absolute floor.  Callers pass a looser norm bound only for the fp32 FMA
+    forward at alpha = 1e-2 (its chain of K sequential roundings per logit is
+    amplified by 1/(2 eps_fd))."""
     e = fd_errors(got, ref)
     assert e["violations"] == 0, (what, e)
     assert e["norm_rel"] <= norm_tol, (what, e)

@@ -114,6 +114,36 @@ def test_meta_grad_parity_wide_dims_small_batch(gemm_mode):
     check(W.CONFIGS["wide4096"].dims, 48, 0, gemm_mode=gemm_mode)
 
 
+def test_meta_grad_parity_on_the_paths_full_size_models_take():
+    """A shape that takes what the 4096-wide model takes at its full batch, at a cost the CPU checker pays in
+    seconds: batch x widest layer = 6 Mi elements, so the chain's small kernels run without dependent-launch
+    overlap, and the first layer's forward product (1536 x 4096 x 512) is 96 CTA-pair tiles on 74 resident
+    pairs, so its last 22 tiles are each shared by two pairs.  Both forward modes against one checker run."""
+    dims, batch = (512, 4096, 32), 1536
+    cached = {}
+    for gemm_mode in (2, 1):
+        cfg, w = W.custom_mlp(dims, batch, seed=17)
+        if not cached:
+            theta = (w["theta"] + 0.05 * W.normal(17, 99, cfg.n_params).astype(np.float32)).astype(np.float32)
+            cached["theta"] = away_from_kinks(dims, theta, w["X"])
+            cached["ref"] = oracle.meta_grad(dims, cached["theta"], w["X"], w["y_clean"])
+        theta, (loss_ref, g_ref) = cached["theta"], cached["ref"]
+        with Ctx(cfg.n_params, batch, dims, gemm_mode) as ctx:
+            g = torch.full((cfg.n_params,), float("nan"), dtype=torch.float32, device=DEV)
+            loss = torch.zeros(1, dtype=torch.float32, device=DEV)
+            B.sama_meta_grad(ctx.h, ctx.mlp, dev(theta), dev(w["X"]), dev(w["y_clean"]), batch, g, loss)
+            torch.cuda.synchronize()
+            assert B.sama_device_status(ctx.h) == 0
+            g1 = g.cpu().numpy()
+        assert float(loss.item()) == pytest.approx(loss_ref, rel=2e-5)
+        worst = 0.0
+        for a, b in blocks(dims):
+            scale = np.abs(g_ref[a:b]).max()
+            worst = max(worst, float(np.abs(g1[a:b] - g_ref[a:b]).max() / scale))
+        print("\n[meta_grad] dims=%s B=%d gemm_mode=%d: worst block-relative error %.2e" % (dims, batch, gemm_mode, worst))
+        assert worst <= 5e-5, worst
+
+
 def test_meta_grad_feeds_the_step():
     """The whole chain on the device: g_meta from a clean batch, then the SAMA step on the noisy batch."""
     cfg = W.CONFIGS["tiny"]

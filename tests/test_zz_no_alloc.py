@@ -1,9 +1,10 @@
-"""The allocation-free adaptation entry point against the regular one.
+"""The allocation-free adaptation entry point against the regular one and against the CPU checker.
 
 ``sama_adapt_noalloc`` is for callers that are not allowed to call cudaMalloc
 (code under a framework allocator that owns the device, plug-ins loaded after
 memory pools were frozen): it keeps the reduction scratch in a static device
-array instead of a context.  It must give what ``sama_adapt`` gives.  The file
+array instead of a context.  It must give what ``sama_adapt`` gives (and what the CPU
+checker gives for Eq. 4 / Appendix C), and a call must leave the device's free memory where it was.  The file
 name sorts last so that a run stopping at the first failure has already run
 everything else; the test also passes on its own in a fresh process.
 """
@@ -11,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2310_05674_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
@@ -31,6 +33,19 @@ def test_noalloc_adapt_matches_context_adapt_twice_in_a_row():
         ss_new = torch.full((1,), -1.0, dtype=torch.float64, device=dev)
         B.sama_adapt_noalloc(n, t["m"], t["s"], gb, t["g_meta"], adam, p_new, ss_new)
         torch.cuda.synchronize()
+        # the name's promise: a further call (the set-up of the first one is done) moves no device memory
+        free_before = torch.cuda.mem_get_info(0)[0]
+        B.sama_adapt_noalloc(n, t["m"], t["s"], gb, t["g_meta"], adam, p_new, ss_new)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info(0)[0] == free_before
+        # against the CPU checker (same fp32-rounded hyper-parameters as the C ABI receives)
+        f = lambda x: float(np.float32(x))
+        ref = oracle.adapt(w["m"], w["s"], w["g_base"] if use_g else None, w["g_meta"],
+                           oracle.Adam(f(adam.lr), f(adam.beta1), f(adam.beta2), f(adam.eps), adam.step))
+        got = p_new.cpu().numpy().astype(np.float64)
+        scale = np.maximum(np.abs(ref), 1e-3 * np.abs(ref).max())
+        assert float((np.abs(got - ref) / scale).max()) <= 1e-5
+        assert float(ss_new.item()) == pytest.approx(oracle.sumsq(ref), rel=2e-6)
         results.append((n, adam, t, gb, p_new, ss_new))
     ctx = B.sama_create(0, max(r[0] for r in results), 0, None)
     try:
