@@ -3,12 +3,19 @@
 
 One "step" is one pass of the whole path -- adaptation + norm, perturbation,
 dual-branch forward, cross-entropy + central difference -- over one synthetic
-batch.  Prints ONE JSON line (rank 0).  ``--impl reference`` times the CPU
-checker on the host cores instead (rank 0 only).
+batch.  Prints ONE JSON line (rank 0).  The line's headline (value, roofline,
+e2e, cpu_baseline) is the largest single-GPU workload, the 4096-wide MLP; with
+one GPU the same line also carries, under "workloads", the other MLP workloads
+(steps/s, forward fraction of roofline) and the adaptation + perturbation sweep
+on the 110 M / 355 M flat vectors (HBM GB/s).  ``--impl reference`` times the
+CPU checker on the host cores instead (rank 0 only).
 
 Timing: CUDA events on the launching stream around each step, an L2 flush
 (a write larger than L2) between steps outside the events, W >= 3 warm-ups,
-barrier + synchronize on both sides, max over ranks.
+barrier + synchronize on both sides, max over ranks.  ``--steps K`` is
+multiplied inside: every one of the K steps is repeated ``inner_reps`` times
+(each repetition timed by its own event pair) so that the timed region lasts
+about a second and the clock sampler sees it; rates are per single step.
 """
 from __future__ import annotations
 
@@ -180,6 +187,22 @@ class OracleTimer:
         return t, desc
 
 
+PRIMARY = "wide4096"
+EXTRAS = ["mlp3072", "head1024", "tiny", "flat355m", "flat110m"]
+
+
+def config_for(name: str, flat_n: int = 0) -> dict:
+    """The workload description both arms print (identical dicts)."""
+    if name in W.FLAT_SIZES:
+        return {"workload": name, "dims": None, "batch": 0, "n_params": int(flat_n or W.FLAT_SIZES[name]),
+                "alpha": 1.0, "l2": "flushed between steps (256 MiB write, outside the events)",
+                "replicas": "one independent step per rank, no data-path collective"}
+    cfg = W.CONFIGS[name]
+    return {"workload": name, "dims": list(cfg.dims), "batch": cfg.batch, "n_params": cfg.n_params,
+            "alpha": cfg.alpha, "l2": "flushed between steps (256 MiB write, outside the events)",
+            "replicas": "one independent step per rank, no data-path collective"}
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -187,7 +210,7 @@ def run_reference(args):
     name = args.workload
     flat = name in W.FLAT_SIZES
     cfg = None if flat else W.CONFIGS[name]
-    w = W.flat_vector(W.FLAT_SIZES[name], 0) if flat else W.mlp_workload(cfg, 0)
+    w = W.flat_vector(args.flat_n or W.FLAT_SIZES[name], 0) if flat else W.mlp_workload(cfg, 0)
     timer = OracleTimer(name, w, cfg)
     budget = 150.0 / max(1, args.steps + args.warmup)
     times, desc = [], ""
@@ -201,23 +224,315 @@ def run_reference(args):
            "unit": "steps/s", "n_gpus": args.gpus,
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": name},
+           "config": config_for(name, args.flat_n),
            "cpu_baseline": {"value": value, "unit": "steps/s", "cores": 1, "kind": "oracle",
                             "sample": "each step: " + desc},
            "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(out), flush=True)
 
 
+class Bench:
+    """Shared state of one rank's measurements: device, replica group, peaks, the L2-flush buffer."""
+
+    def __init__(self, args):
+        import torch
+        from paper_2310_05674_b200 import binding as S
+        from paper_2310_05674_b200 import replicas
+        self.torch, self.S, self.args = torch, S, args
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        torch.cuda.set_device(self.local)
+        self.dev = "cuda:%d" % self.local
+        self.group = replicas.init(backend="nccl", device=self.dev)   # one process per GPU; independent replicas
+        self.peaks = load_peaks()
+        self.flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=self.dev)
+        self.stream = torch.cuda.current_stream()
+        self.sm_count = torch.cuda.get_device_properties(self.local).multi_processor_count
+
+    def barrier(self):
+        self.group.barrier()
+        self.torch.cuda.synchronize()
+
+    def tensor_peaks(self):
+        """fp32-faithful tensor-core peak: dense TF32 = measured bf16 x 0.5 (nominal ratio), three products per
+        fp32 product.  Burst for a kernel timed at full clock, sustained under the board's power cap."""
+        p = self.peaks
+        return p["bf16_tflops"] * 0.5 / 3.0, p["bf16_tflops_sustained"] * 0.5 / 3.0
+
+    def measure(self, name, w, region_s, with_e2e=False, with_meta=False, flat_n=0):
+        """Times one workload: W warm-ups, then K x inner_reps steps, each between its own pair of events."""
+        torch, S, args = self.torch, self.S, self.args
+        dev, stream, group = self.dev, self.stream, self.group
+        flat = name in W.FLAT_SIZES
+        cfg = None if flat else W.CONFIGS[name]
+        n = w["theta"].size
+        mlp = None if flat else S.MLP(cfg.dims)
+        B = cfg.batch if cfg else 0
+        ctx = S.sama_create(self.local, n, B, mlp)
+        if args.gemm_mode:
+            S.sama_set_gemm_mode(ctx, args.gemm_mode)
+        adam = S.Adam()
+        alpha = cfg.alpha if cfg else 1.0
+        keys = ["theta", "m", "s", "g_base", "g_meta"] + ([] if flat else ["X", "y", "lam"])
+        pin = with_e2e and not flat
+        host = {k: torch.from_numpy(np.ascontiguousarray(w[k])) for k in keys}
+        if pin:
+            host = {k: v.pin_memory() for k, v in host.items()}
+        d = {k: host[k].to(dev) for k in keys}
+        p, tp, tm = (torch.empty(n, dtype=torch.float32, device=dev) for _ in range(3))
+        mg = torch.empty(max(B, 1), dtype=torch.float32, device=dev)
+        flush_buf = self.flush_buf
+
+        outputs = {"plus": tp, "minus": tm}
+
+        def one_step():
+            if flat:
+                S.sama_adapt(ctx, n, d["m"], d["s"], d["g_base"], d["g_meta"], adam, p, None, stream)
+                S.sama_perturb(ctx, n, d["theta"], p, S.sama_ctx_sumsq(ctx), alpha, tp, tm, None, stream)
+            else:
+                S.sama_step(ctx, mlp, n, d["theta"], d["m"], d["s"], d["g_base"], d["g_meta"], adam, alpha, d["X"],
+                            d["y"], d["lam"], B, p, outputs["plus"], outputs["minus"], mg, None, None, stream)
+
+        def timed(K):
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+            for a, b in ev:
+                flush_buf.fill_(1)
+                a.record(stream)
+                one_step()
+                b.record(stream)
+            torch.cuda.synchronize()
+            return [a.elapsed_time(b) for a, b in ev]
+
+        sampler = ClockSampler(self.local)
+        sampler.start()
+        for _ in range(args.warmup):
+            flush_buf.fill_(1)
+            one_step()
+        torch.cuda.synchronize()
+        # inner repetitions: enough for the timed region to last about region_s (every rank takes the same count)
+        est_ms = max(group.max_over_ranks(sum(timed(3)) / 3.0, dev), 1e-3)
+        reps = int(min(max(1, round(region_s * 1e3 / (est_ms * args.steps))), 4096))
+        total_steps = args.steps * reps
+        self.barrier()
+        l0 = S.sama_launch_count(ctx)
+        sampler.active.set()
+        t_wall0 = time.perf_counter()
+        ms = timed(total_steps)
+        self.barrier()
+        t_wall = time.perf_counter() - t_wall0
+        sampler.active.clear()
+        launches = S.sama_launch_count(ctx) - l0
+        total_ms = group.max_over_ranks(sum(ms), dev)
+        ms_per_step = total_ms / total_steps
+        value = group.world * total_steps / (total_ms * 1e-3)
+        status = S.sama_device_status(ctx)
+        clocks = sampler.summary()
+
+        # ---- per-kernel times (events recorded by the library around each launch, same stream) ----
+        S.sama_profile_enable(ctx, True)
+        Kp = min(total_steps, 50)
+        sampler.active.set()
+        timed(Kp)
+        sampler.active.clear()
+        recs = S.sama_profile_collect(ctx)
+        per_kernel = {}
+        for kind, layer, t in recs:
+            key = S.KERNEL_KINDS.get(kind, str(kind))
+            e = per_kernel.setdefault(key, {"ms_per_step": 0.0, "launches_per_step": 0.0, "layers": {}})
+            e["ms_per_step"] += t / Kp
+            e["launches_per_step"] += 1.0 / Kp
+            if layer >= 0:
+                e["layers"][layer] = e["layers"].get(layer, 0.0) + t / Kp
+        # second pass, grouped: the forward layers of a step between ONE pair of events (an event between two
+        # launches serialises them and removes the dependent-launch overlap they have in an untimed step)
+        S.sama_profile_enable(ctx, 2)
+        sampler.active.set()
+        timed(Kp)
+        sampler.active.clear()
+        grouped = {}
+        for kind, layer, t, run_len in S.sama_profile_collect(ctx, with_launches=True):
+            key = S.KERNEL_KINDS.get(kind, str(kind))
+            e = grouped.setdefault(key, {"ms_per_step": 0.0, "launches_per_step": 0.0})
+            e["ms_per_step"] += t / Kp
+            e["launches_per_step"] += run_len / Kp
+        S.sama_profile_enable(ctx, 0)
+        for key, e in grouped.items():
+            if key in per_kernel and key.startswith("gemm"):
+                per_kernel[key]["ms_per_step_per_launch_events"] = per_kernel[key]["ms_per_step"]
+                per_kernel[key]["ms_per_step"] = e["ms_per_step"]
+                per_kernel[key]["timing"] = "one event pair around the step's consecutive launches of this kernel"
+        dominant = max(per_kernel, key=lambda k: per_kernel[k]["ms_per_step"])
+        peaks = self.peaks
+        power_capped = "sw_power_cap" in clocks["reasons"] or (
+            clocks["sm_mhz"] and clocks["sm_max_mhz"] and clocks["sm_mhz"] < 0.9 * clocks["sm_max_mhz"])
+
+        def launch_s(kernel):
+            return per_kernel[kernel]["ms_per_step"] / max(per_kernel[kernel]["launches_per_step"], 1e-9) * 1e-3
+
+        def hbm_roof(kernel, bytes_per_launch, seconds=None, moved=None):
+            t = seconds if seconds is not None else launch_s(kernel)
+            ach = bytes_per_launch / t / 1e9
+            r = {"bound": "hbm", "kernel": kernel, "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                 "frac": ach / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
+                 "frac_of_nominal_8TBs": ach / 8000.0, "traffic": recorded_traffic(kernel, name),
+                 "algorithmic_bytes_per_launch": bytes_per_launch, "launch_us": t * 1e6}
+            if moved is not None:   # bytes the kernel moves including the forward's operand preparation (L2 and HBM)
+                r["bytes_moved_incl_operand_prep"] = moved
+                r["moved_gbs"] = moved / t / 1e9
+            return r
+
+        rooflines = {}
+        if "adapt_sumsq" in per_kernel:
+            rooflines["adapt_sumsq"] = hbm_roof("adapt_sumsq", 20.0 * n)
+        if "perturb" in per_kernel:
+            rooflines["perturb"] = hbm_roof("perturb", 16.0 * n)
+        if "perturb_split" in per_kernel:
+            # the perturbation of Sec. 3.2 is 16 B/element (theta, p in; theta+, theta- out); what the same sweep
+            # also writes for the tensor-core forward (hi / lo of W+-: 32 B/element unless theta+- are not
+            # stored, and the split of X) is operand preparation, reported beside it
+            moved = (40.0 if self.store_theta_pm else 32.0) * n + (12.0 * B * cfg.dims[0] if cfg else 0.0)
+            rooflines["perturb_split"] = hbm_roof("perturb_split", 16.0 * n, moved=moved)
+        if "fused_sweep" in per_kernel:   # adaptation + norm + perturbation (+ operand split) in one launch
+            moved = (44.0 if self.store_theta_pm else 36.0) * n + 16.0 * n + (12.0 * B * cfg.dims[0] if cfg else 0.0)
+            rooflines["fused_sweep"] = hbm_roof("fused_sweep", 36.0 * n, moved=moved)
+        sweep = [k for k in ("adapt_sumsq", "perturb", "perturb_split", "sumsq", "fused_sweep") if k in per_kernel]
+        if sweep:   # adaptation + norm + perturbation together: 36 B/element over the sum of their launch times
+            t = sum(per_kernel[k]["ms_per_step"] for k in sweep) * 1e-3
+            rooflines["adapt_perturb"] = hbm_roof("+".join(sweep), 36.0 * n, seconds=t)
+        for gk in ("gemm_ffma", "gemm_tf32x3"):
+            if gk in per_kernel and cfg:
+                flops = float(cfg.forward_flops)
+                t = per_kernel[gk]["ms_per_step"] * 1e-3
+                ach = flops / t / 1e12
+                if gk == "gemm_ffma":
+                    mhz = clocks["sm_mhz"] or clocks["sm_max_mhz"] or 1965.0
+                    peak = self.sm_count * FMA_LANES_PER_SM * 2 * mhz * 1e6 / 1e12
+                    rooflines[gk] = {"bound": "alu", "kernel": gk, "achieved": ach, "peak": peak, "unit": "TFLOP/s",
+                                     "frac": ach / peak,
+                                     "peak_source": "%d SMs x 128 FMA lanes x 2 x %.0f MHz (median SM clock sampled "
+                                                    "during the run)" % (self.sm_count, mhz),
+                                     "traffic": recorded_traffic(gk, name), "algorithmic_flops_per_step": flops}
+                else:
+                    burst, sustained = self.tensor_peaks()
+                    peak = sustained if power_capped else burst
+                    rooflines[gk] = {"bound": "tensor", "kernel": gk, "achieved": ach, "peak": peak,
+                                     "unit": "TFLOP/s", "frac": ach / peak,
+                                     "regime": "sustained (power cap or reduced clock seen)" if power_capped
+                                               else "burst (full clock, no cap)",
+                                     "frac_of_burst_peak": ach / burst, "frac_of_sustained_peak": ach / sustained,
+                                     "peak_source": peaks["source"] + " bf16 (burst %.1f / sustained %.1f TFLOP/s) x 0.5 "
+                                                    "(nominal tf32:bf16) / 3 products per fp32-faithful product"
+                                                    % (peaks["bf16_tflops"], peaks["bf16_tflops_sustained"]),
+                                     "traffic": recorded_traffic(gk, name), "algorithmic_flops_per_step": flops,
+                                     "launches_per_step": per_kernel[gk]["launches_per_step"]}
+        roofline = rooflines.get(dominant) or next(iter(rooflines.values()))
+
+        out = {"value": value, "unit": "steps/s", "ms_per_step": ms_per_step, "steps": args.steps,
+               "inner_reps": reps, "timed_steps": total_steps, "config": config_for(name, flat_n),
+               "clocks": clocks, "gpu_launches": int(launches), "device_status": int(status),
+               "forward_path": {0: "none", 1: "fp32 FMA", 2: "tensor cores, 3xTF32"}[S.sama_last_forward_path(ctx)],
+               "wall_s_timed_region": t_wall, "roofline": roofline, "rooflines": rooflines, "kernels": per_kernel}
+        if flat:
+            out["adapt_perturb_gbs"] = 36.0 * n / (ms_per_step * 1e-3) / 1e9
+
+        # ---- the same step for a caller that keeps only what the method hands on: the meta gradient and the nudged
+        # base parameters theta- (Sec. 3.2); theta+ is not requested, so the sweep never writes it ----
+        if not flat:
+            outputs["plus"] = None
+            Kv = min(total_steps, 200)
+            for _ in range(3):
+                flush_buf.fill_(1)
+                one_step()
+            msv = sum(timed(Kv)) / Kv
+            S.sama_profile_enable(ctx, 1)
+            timed(min(Kv, 20))
+            pv = {}
+            for kind, layer, t in S.sama_profile_collect(ctx):
+                key = S.KERNEL_KINDS.get(kind, str(kind))
+                pv[key] = pv.get(key, 0.0) + t / min(Kv, 20)
+            S.sama_profile_enable(ctx, 0)
+            outputs["plus"] = tp
+            out["without_theta_plus_output"] = {"value": group.world * 1e3 / group.max_over_ranks(msv, dev), "unit": "steps/s",
+                                                "ms_per_step": msv, "steps": Kv, "kernels": pv}
+
+        # ---- end to end through the host-buffer entry point ----
+        if with_e2e and not flat and not args.no_e2e:
+            mg_h = torch.empty(B, dtype=torch.float32).pin_memory()
+            eps_h = torch.empty(1, dtype=torch.float32).pin_memory()
+            Ke = max(3, min(args.steps, 30))
+
+            def host_step():
+                S.sama_step_host(ctx, mlp, n, host["theta"], host["m"], host["s"], host["g_base"], host["g_meta"],
+                                 adam, alpha, host["X"], host["y"], host["lam"], B, mg_h, eps_h, None, stream)
+            for _ in range(3):
+                host_step()
+            self.barrier()
+            t0 = time.perf_counter()
+            for _ in range(Ke):
+                host_step()
+            self.barrier()
+            te = group.max_over_ranks(time.perf_counter() - t0, dev)
+            h2d = sum(host[k].numel() * host[k].element_size() for k in keys)
+            out["e2e"] = {"value": group.world * Ke / te, "unit": "steps/s", "h2d_bytes_per_step": int(h2d),
+                          "d2h_bytes_per_step": int(4 * B + 4), "steps": Ke,
+                          "note": "sama_step_host: all inputs copied from pinned host memory every step"}
+        if with_meta and not flat:
+            gm_out = torch.empty(n, dtype=torch.float32, device=dev)
+            for _ in range(3):
+                S.sama_meta_grad(ctx, mlp, d["theta"], d["X"], d["y"], B, gm_out, None, stream)
+            Km = max(3, min(args.steps, 50))
+            evm = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(Km)]
+            for a_, b_ in evm:
+                flush_buf.fill_(1)
+                a_.record(stream)
+                S.sama_meta_grad(ctx, mlp, d["theta"], d["X"], d["y"], B, gm_out, None, stream)
+                b_.record(stream)
+            torch.cuda.synchronize()
+            msm = sum(a_.elapsed_time(b_) for a_, b_ in evm) / Km
+            flops_m = 1.5 * cfg.forward_flops   # forward + dz W + dz^T h of ONE branch = 3/2 of the dual-branch forward
+            if args.gemm_mode == 1:
+                mhz = clocks["sm_mhz"] or 1965.0
+                peak_m = self.sm_count * FMA_LANES_PER_SM * 2 * mhz * 1e6 / 1e12
+                bound_m, src_m = "alu", "%d SMs x 128 FMA lanes x 2 x %.0f MHz" % (self.sm_count, mhz)
+            else:
+                peak_m = self.tensor_peaks()[1]
+                bound_m, src_m = "tensor", peaks["source"] + " sustained bf16 x 0.5 / 3 products per fp32-faithful product"
+            ach_m = flops_m / (msm * 1e-3) / 1e12
+            out["meta_grad"] = {"ms_per_call": msm, "calls_per_s": 1e3 / msm, "bound": bound_m, "achieved": ach_m,
+                                "peak": peak_m, "unit": "TFLOP/s", "frac": ach_m / peak_m, "peak_source": src_m,
+                                "note": "algorithmic flops = 3 single-branch matrix products per layer (forward, "
+                                        "dz W, dz^T h); time includes the operand split / transpose kernels"}
+        sampler.stop_flag.set()
+        S.sama_destroy(ctx)
+        del d, p, tp, tm, host
+        torch.cuda.empty_cache()
+        return out
+
+    store_theta_pm = True   # the benchmark asks sama_step for theta+ and theta- (the paper's nudge uses theta-)
+
+
+def brief(r):
+    """What the line keeps of a secondary workload."""
+    keep = {k: r[k] for k in ("value", "unit", "ms_per_step", "inner_reps", "timed_steps", "clocks", "forward_path",
+                              "device_status", "adapt_perturb_gbs", "without_theta_plus_output") if k in r}
+    keep["rooflines"] = r["rooflines"]
+    keep["kernels"] = {k: round(v["ms_per_step"], 6) for k, v in r["kernels"].items()}
+    keep["gemm_layers_ms"] = {k: v["layers"] for k, v in r["kernels"].items() if k.startswith("gemm")}
+    return keep
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="mlp3072", choices=sorted(W.CONFIGS) + sorted(W.FLAT_SIZES))
+    ap.add_argument("--workload", default=PRIMARY, choices=sorted(W.CONFIGS) + sorted(W.FLAT_SIZES))
     ap.add_argument("--gemm-mode", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="time only --workload (the other workloads are added by default on one GPU)")
+    ap.add_argument("--region-s", type=float, default=1.2, help="target length of the primary timed region")
     ap.add_argument("--flat-n", type=int, default=0, help="override the length of a flat-vector workload")
     ap.add_argument("--meta-grad", action="store_true",
                     help="also time sama_meta_grad (the direct gradient that produces g_meta) on the same batch")
@@ -228,226 +543,60 @@ def main():
         run_reference(args)
         return
 
-    import torch
-    from paper_2310_05674_b200 import binding as S
-    from paper_2310_05674_b200 import replicas
-
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dev = "cuda:%d" % local
-    group = replicas.init(backend="nccl", device=dev)   # one process per GPU; independent replicas
-    world, rank = group.world, group.rank
-
-    def barrier():
-        group.barrier()
-        torch.cuda.synchronize()
-
-    def max_over_ranks(x: float) -> float:
-        return group.max_over_ranks(x, dev)
-
-    peaks = load_peaks()
+    b = Bench(args)
+    world, rank = b.group.world, b.group.rank
     name = args.workload
     flat = name in W.FLAT_SIZES
-    seed = group.seed  # each rank owns an independent batch / vector: no data-path collective
-    if flat:
-        n = args.flat_n or W.FLAT_SIZES[name]
-        w = W.flat_vector(n, seed)
-        cfg = None
-        ctx = S.sama_create(local, n, 0, None)
-        mlp = None
-    else:
-        cfg = W.CONFIGS[name]
-        w = W.mlp_workload(cfg, seed)
-        n = cfg.n_params
-        mlp = S.MLP(cfg.dims)
-        ctx = S.sama_create(local, n, cfg.batch, mlp)
-    if args.gemm_mode:
-        S.sama_set_gemm_mode(ctx, args.gemm_mode)
-    adam = S.Adam()
-    alpha = cfg.alpha if cfg else 1.0
+    seed = b.group.seed  # each rank owns an independent batch / vector: no data-path collective
+    cfg = None if flat else W.CONFIGS[name]
+    w = W.flat_vector(args.flat_n or W.FLAT_SIZES[name], seed) if flat else W.mlp_workload(cfg, seed)
+    r = b.measure(name, w, args.region_s, with_e2e=True, with_meta=args.meta_grad, flat_n=args.flat_n)
 
-    keys = ["theta", "m", "s", "g_base", "g_meta"] + ([] if flat else ["X", "y", "lam"])
-    host = {k: torch.from_numpy(np.ascontiguousarray(w[k])).pin_memory() for k in keys}
-    d = {k: host[k].to(dev) for k in keys}
-    p, tp, tm = (torch.empty(n, dtype=torch.float32, device=dev) for _ in range(3))
-    B = cfg.batch if cfg else 0
-    mg = torch.empty(max(B, 1), dtype=torch.float32, device=dev)
-    flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
-    stream = torch.cuda.current_stream()
-
-    def one_step():
-        if flat:
-            S.sama_adapt(ctx, n, d["m"], d["s"], d["g_base"], d["g_meta"], adam, p, None, stream)
-            S.sama_perturb(ctx, n, d["theta"], p, S.sama_ctx_sumsq(ctx), alpha, tp, tm, None, stream)
-        else:
-            S.sama_step(ctx, mlp, n, d["theta"], d["m"], d["s"], d["g_base"], d["g_meta"], adam, alpha, d["X"],
-                        d["y"], d["lam"], B, p, tp, tm, mg, None, None, stream)
-
-    def timed(K, profile=False):
-        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
-        for a, b in ev:
-            flush_buf.fill_(1)
-            a.record(stream)
-            one_step()
-            b.record(stream)
-        torch.cuda.synchronize()
-        return [a.elapsed_time(b) for a, b in ev]
-
-    sampler = ClockSampler(local)
-    sampler.start()
-
-    for _ in range(args.warmup):
-        flush_buf.fill_(1)
-        one_step()
-    barrier()
-    l0 = S.sama_launch_count(ctx)
-    sampler.active.set()
-    t_wall0 = time.perf_counter()
-    ms = timed(args.steps)
-    barrier()
-    t_wall = time.perf_counter() - t_wall0
-    launches = S.sama_launch_count(ctx) - l0
-    total_ms = max_over_ranks(sum(ms))
-    ms_per_step = total_ms / args.steps
-    value = world * args.steps / (total_ms * 1e-3)
-    status = S.sama_device_status(ctx)
-
-    # ---- per-kernel times (events recorded by the library around each launch, same stream) ----
-    S.sama_profile_enable(ctx, True)
-    Kp = min(args.steps, 50)
-    timed(Kp)
-    recs = S.sama_profile_collect(ctx)
-    S.sama_profile_enable(ctx, False)
-    sampler.active.clear()
-    per_kernel = {}
-    for kind, layer, t in recs:
-        key = S.KERNEL_KINDS.get(kind, str(kind))
-        e = per_kernel.setdefault(key, {"ms_per_step": 0.0, "launches_per_step": 0.0, "layers": {}})
-        e["ms_per_step"] += t / Kp
-        e["launches_per_step"] += 1.0 / Kp
-        if layer >= 0:
-            e["layers"][layer] = e["layers"].get(layer, 0.0) + t / Kp
-    dominant = max(per_kernel, key=lambda k: per_kernel[k]["ms_per_step"])
-    clocks_mid = sampler.summary()
-    sm_count = torch.cuda.get_device_properties(local).multi_processor_count
-
-    def hbm_roof(kernel, bytes_per_launch):
-        t = per_kernel[kernel]["ms_per_step"] / max(per_kernel[kernel]["launches_per_step"], 1e-9) * 1e-3
-        ach = bytes_per_launch / t / 1e9
-        return {"bound": "hbm", "kernel": kernel, "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
-                "frac_of_nominal_8TBs": ach / 8000.0, "traffic": recorded_traffic(kernel, name),
-                "algorithmic_bytes_per_launch": bytes_per_launch}
-
-    rooflines = {}
-    if "adapt_sumsq" in per_kernel:
-        rooflines["adapt_sumsq"] = hbm_roof("adapt_sumsq", 20.0 * n)
-    if "perturb" in per_kernel:
-        rooflines["perturb"] = hbm_roof("perturb", 16.0 * n)
-    if "perturb_split" in per_kernel:  # perturb + TF32 hi/lo of both branches: 8 read + 8 + 16 written per element
-        # ... plus the batch's operand split done by the same sweep: 4 read + 8 written per element of X
-        rooflines["perturb_split"] = hbm_roof("perturb_split", 32.0 * n + (12.0 * B * cfg.dims[0] if cfg else 0.0))
-    for gk in ("gemm_ffma", "gemm_tf32x3"):
-        if gk in per_kernel and cfg:
-            flops = float(cfg.forward_flops)
-            t = per_kernel[gk]["ms_per_step"] * 1e-3
-            ach = flops / t / 1e12
-            if gk == "gemm_ffma":
-                mhz = clocks_mid["sm_mhz"] or clocks_mid["sm_max_mhz"] or 1965.0
-                peak = sm_count * FMA_LANES_PER_SM * 2 * mhz * 1e6 / 1e12
-                rooflines[gk] = {"bound": "alu", "kernel": gk, "achieved": ach, "peak": peak, "unit": "TFLOP/s",
-                                 "frac": ach / peak,
-                                 "peak_source": "%d SMs x 128 FMA lanes x 2 x %.0f MHz (median SM clock sampled "
-                                                "during the run)" % (sm_count, mhz),
-                                 "traffic": recorded_traffic(gk, name), "algorithmic_flops_per_step": flops}
-            else:
-                peak = peaks["bf16_tflops_sustained"] * 0.5 / 3.0
-                rooflines[gk] = {"bound": "tensor", "kernel": gk, "achieved": ach, "peak": peak, "unit": "TFLOP/s",
-                                 "frac": ach / peak,
-                                 "peak_source": peaks["source"] + " sustained bf16 x 0.5 (nominal tf32:bf16) / 3 "
-                                                "products per fp32-faithful product",
-                                 "traffic": recorded_traffic(gk, name), "algorithmic_flops_per_step": flops}
-    roofline = rooflines.get(dominant) or next(iter(rooflines.values()))
-
-    # ---- end to end through the host-buffer entry point ----
-    e2e = None
-    if not flat and not args.no_e2e:
-        mg_h = torch.empty(B, dtype=torch.float32).pin_memory()
-        eps_h = torch.empty(1, dtype=torch.float32).pin_memory()
-        Ke = max(3, min(args.steps, 30))
-
-        def host_step():
-            S.sama_step_host(ctx, mlp, n, host["theta"], host["m"], host["s"], host["g_base"], host["g_meta"], adam,
-                             alpha, host["X"], host["y"], host["lam"], B, mg_h, eps_h, None, stream)
-        for _ in range(3):
-            host_step()
-        barrier()
-        sampler.active.set()
-        t0 = time.perf_counter()
-        for _ in range(Ke):
-            host_step()
-        barrier()
-        te = max_over_ranks(time.perf_counter() - t0)
-        sampler.active.clear()
-        h2d = sum(host[k].numel() * host[k].element_size() for k in keys)
-        e2e = {"value": world * Ke / te, "unit": "steps/s", "h2d_bytes_per_step": int(h2d),
-               "d2h_bytes_per_step": int(4 * B + 4), "steps": Ke,
-               "note": "sama_step_host: all inputs copied from pinned host memory every step"}
-    meta = None
-    if args.meta_grad and not flat:
-        gm_out = torch.empty(n, dtype=torch.float32, device=dev)
-        for _ in range(3):
-            S.sama_meta_grad(ctx, mlp, d["theta"], d["X"], d["y"], B, gm_out, None, stream)
-        Km = max(3, min(args.steps, 50))
-        evm = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(Km)]
-        sampler.active.set()
-        for a_, b_ in evm:
-            flush_buf.fill_(1)
-            a_.record(stream)
-            S.sama_meta_grad(ctx, mlp, d["theta"], d["X"], d["y"], B, gm_out, None, stream)
-            b_.record(stream)
-        torch.cuda.synchronize()
-        sampler.active.clear()
-        msm = sum(a_.elapsed_time(b_) for a_, b_ in evm) / Km
-        flops_m = 1.5 * cfg.forward_flops   # forward + dz W + dz^T h of ONE branch = 3/2 of the dual-branch forward
-        if args.gemm_mode == 1:
-            mhz = (sampler.summary()["sm_mhz"] or 1965.0)
-            peak_m = sm_count * FMA_LANES_PER_SM * 2 * mhz * 1e6 / 1e12
-            bound_m, src_m = "alu", "%d SMs x 128 FMA lanes x 2 x %.0f MHz" % (sm_count, mhz)
-        else:
-            peak_m = peaks["bf16_tflops_sustained"] * 0.5 / 3.0
-            bound_m, src_m = "tensor", peaks["source"] + " sustained bf16 x 0.5 / 3 products per fp32-faithful product"
-        ach_m = flops_m / (msm * 1e-3) / 1e12
-        meta = {"ms_per_call": msm, "calls_per_s": 1e3 / msm, "bound": bound_m, "achieved": ach_m, "peak": peak_m,
-                "unit": "TFLOP/s", "frac": ach_m / peak_m, "peak_source": src_m,
-                "note": "algorithmic flops = 3 single-branch matrix products per layer (forward, dz W, dz^T h); "
-                        "time includes the operand split / transpose kernels"}
-    sampler.stop_flag.set()
-    clocks = sampler.summary()
-
-    out = {"metric": METRIC if not flat else "adapt+perturb sweeps/sec", "value": value, "unit": "steps/s",
-           "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
-           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-           "config": {"workload": name, "dims": list(cfg.dims) if cfg else None, "batch": B, "n_params": n,
-                      "alpha": alpha, "l2": "flushed between steps (256 MiB write, outside the events)",
-                      "replicas": "one independent step per rank, no data-path collective"},
-           "clocks": clocks, "gpu_launches": int(launches), "device_status": int(status),
-           "wall_s_timed_region": t_wall, "roofline": roofline, "rooflines": rooflines, "kernels": per_kernel}
-    if meta:
-        out["meta_grad"] = meta
-    if e2e:
-        out["e2e"] = e2e
-    if flat:
-        out["adapt_perturb_gbs"] = 36.0 * n / (ms_per_step * 1e-3) / 1e9
+    out = {"metric": METRIC if not flat else "adapt+perturb sweeps/sec", "value": r["value"], "unit": "steps/s",
+           "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": r["ms_per_step"],
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic"}
+    for k in ("inner_reps", "timed_steps", "config", "clocks", "gpu_launches", "device_status", "forward_path",
+              "wall_s_timed_region", "roofline", "rooflines", "kernels", "meta_grad", "e2e", "adapt_perturb_gbs",
+              "without_theta_plus_output"):
+        if k in r:
+            out[k] = r[k]
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         sec, desc = OracleTimer(name, w, cfg).step_seconds(20.0)
         out["cpu_baseline"] = {"value": 1.0 / sec, "unit": "steps/s", "cores": 1, "kind": "oracle", "sample": desc,
                                "host_cores_available": os.cpu_count()}
-    S.sama_destroy(ctx)
+    del w
+
+    # ---- the metric's other configurations (one GPU only: the scaling runs time the headline workload) ----
+    if world == 1 and not args.no_extras and name == PRIMARY:
+        extras = {}
+        flat_w = None
+        for ex in EXTRAS:
+            if ex in W.FLAT_SIZES:
+                nx = W.FLAT_SIZES[ex]
+                if flat_w is None or flat_w["theta"].size < nx:
+                    flat_w = W.flat_vector(nx, seed)
+                # the generator is counter-based: a prefix of the longer vector IS the shorter workload
+                wx = {k: v[:nx] for k, v in flat_w.items()}
+            else:
+                wx = W.mlp_workload(W.CONFIGS[ex], seed)
+            extras[ex] = brief(b.measure(ex, wx, 0.6))
+            del wx
+        out["workloads"] = extras
+        # the metric's three parts in one place
+        out["summary"] = {
+            "steps_per_s": dict([(PRIMARY, r["value"])] + [(k, v["value"]) for k, v in extras.items()
+                                                           if k not in W.FLAT_SIZES]),
+            "adapt_perturb_hbm_gbs": {k: v["adapt_perturb_gbs"] for k, v in extras.items() if k in W.FLAT_SIZES},
+            "adapt_perturb_frac_of_measured_hbm": {k: v["rooflines"]["adapt_perturb"]["frac"] for k, v in extras.items()
+                                                  if k in W.FLAT_SIZES},
+            "forward_frac_of_roofline": dict(
+                [(PRIMARY, r["rooflines"].get("gemm_tf32x3", r["rooflines"].get("gemm_ffma", {})).get("frac"))] +
+                [(k, v["rooflines"].get("gemm_tf32x3", v["rooflines"].get("gemm_ffma", {})).get("frac"))
+                 for k, v in extras.items() if k in ("mlp3072", "head1024")])}
     if rank == 0:
         print(json.dumps(out), flush=True)
-    group.close()
+    b.group.close()
 
 
 if __name__ == "__main__":

@@ -1,8 +1,10 @@
 """Host-side plumbing for running independent replicas of the step, one process per GPU.
 
-The meta-gradient step does not shard in this library: each rank owns a whole
+The per-sample-weight step does not shard in this library: each rank owns a whole
 problem (its own seeded batch and parameter vector) and there is no data-path
-collective.  What the ranks share is only measurement: a barrier on both sides
+collective.  With a shared meta learner (Sec. 4.1) the ranks' dim(lambda)-sized
+meta gradients are combined by one all-reduce per meta step (Sec. 3.3, Fig. 2):
+all_reduce_sum / all_reduce_mean below.  What the ranks otherwise share is only measurement: a barrier on both sides
 of a timed region, the maximum of a duration over ranks, and the aggregate
 throughput (units processed by all ranks divided by that maximum).  The same
 code runs over NCCL on GPUs and over gloo on CPU (which is how it is tested).
@@ -39,6 +41,24 @@ class Replicas:
         t = torch.tensor([float(x)], dtype=torch.float64, device=device)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
+
+    def all_reduce_sum(self, t):
+        """In-place sum of a tensor over ranks: the one gradient synchronisation of the data-parallel step
+        (Sec. 3.3).  With a shared meta learner every rank computes the central difference of Eq. 5 on its own
+        rows of the base batch with the whole batch's size as the normaliser (the B_norm argument of
+        sama_fd_metagrad_reweight), and this sum of the ranks' dim(lambda)-sized vectors is the batch's meta gradient."""
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        return t
+
+    def all_reduce_mean(self, t):
+        """In-place mean over ranks: for ranks that each ran the whole step on their own batch (and their own direct
+        gradient), the way the paper's data-parallel runs average per-replica meta gradients."""
+        self.all_reduce_sum(t)
+        if self.world > 1:
+            t /= self.world
+        return t
 
     def aggregate_rate(self, units_per_rank: float, seconds_this_rank: float, device: str = "cpu") -> float:
         """Whole-job throughput: all ranks' units over the slowest rank's time."""

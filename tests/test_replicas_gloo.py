@@ -70,3 +70,54 @@ def test_single_process_needs_no_group():
         r.close()
     finally:
         os.environ.update(env)
+
+
+CHILD_SYNC = textwrap.dedent("""
+    import json, sys
+    sys.path.insert(0, %r)
+    import numpy as np, torch
+    import oracle
+    from paper_2310_05674_b200 import replicas
+    r = replicas.init(backend="gloo")
+    rng = np.random.default_rng(0)                       # the same batch on both ranks; each takes its rows
+    B, H = 24, 5
+    lp = np.abs(rng.normal(size=B)) + 0.1
+    lm = lp * (1 + 1e-3 * rng.normal(size=B))
+    lam = (0.5 * rng.normal(size=3 * H + 1)).astype(np.float32)
+    rows = slice(r.rank * B // r.world, (r.rank + 1) * B // r.world)
+    local = oracle.fd_reweight(lp[rows], lm[rows], lam, 0.05, B_norm=B)   # the whole batch's normaliser
+    t = torch.from_numpy(local.copy())
+    r.all_reduce_sum(t)
+    full = oracle.fd_reweight(lp, lm, lam, 0.05, B_norm=B)
+    m = torch.from_numpy(local.copy())
+    r.all_reduce_mean(m)
+    out = {"rank": r.rank, "err": float(np.abs(t.numpy() - full).max() / np.abs(full).max()),
+           "mean_err": float(np.abs(m.numpy() * r.world - full).max() / np.abs(full).max()),
+           "local_differs": bool(np.abs(local - full).max() > 0)}
+    r.barrier()
+    r.close()
+    print("RESULT " + json.dumps(out), flush=True)
+""") % ROOT
+
+
+def test_one_gradient_synchronisation_gives_the_batch_meta_gradient(tmp_path):
+    """Sec. 3.3 / Fig. 2 on CPU with two gloo ranks: each rank's central difference over its own rows (normalised
+    by the whole batch), summed once over ranks, is the central difference over the whole batch."""
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    script = tmp_path / "child_sync.py"
+    script.write_text(CHILD_SYNC)
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE="2",
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env, stdout=subprocess.PIPE,
+                                      stderr=subprocess.PIPE, text=True))
+    import json
+    for p in procs:
+        out, err = p.communicate(timeout=180)
+        assert p.returncode == 0, err[-2000:]
+        d = json.loads([l for l in out.splitlines() if l.startswith("RESULT ")][0][7:])
+        assert d["err"] < 1e-10 and d["mean_err"] < 1e-10 and d["local_differs"]
