@@ -111,7 +111,7 @@ def source_hash(*names):
     return h.hexdigest()[:16]
 
 
-KERNEL_SOURCES = {"adapt_sumsq": ("adapt_perturb.cu",), "perturb": ("adapt_perturb.cu",), "sumsq": ("adapt_perturb.cu",),
+KERNEL_SOURCES = {"fused_sweep": ("adapt_perturb.cu",), "adapt_sumsq": ("adapt_perturb.cu",), "perturb": ("adapt_perturb.cu",), "sumsq": ("adapt_perturb.cu",),
                   "perturb_split": ("adapt_perturb.cu",), "head_ce_fd": ("head_ce_fd.cu",),
                   "gemm_ffma": ("gemm_ffma.cu",), "ce_fd": ("ce_fd.cu",), "gemm_tf32x3": ("gemm_tf32x3.cu",),
                   "split_tf32": ("gemm_tf32x3.cu",)}
@@ -436,7 +436,7 @@ class Bench:
 
         # ---- the same step for a caller that keeps only what the method hands on: the meta gradient and the nudged
         # base parameters theta- (Sec. 3.2); theta+ is not requested, so the sweep never writes it ----
-        if not flat:
+        if not flat and not args.no_variants:
             outputs["plus"] = None
             Kv = min(total_steps, 200)
             for _ in range(3):
@@ -453,6 +453,31 @@ class Bench:
             outputs["plus"] = tp
             out["without_theta_plus_output"] = {"value": group.world * 1e3 / group.max_over_ranks(msv, dev), "unit": "steps/s",
                                                 "ms_per_step": msv, "steps": Kv, "kernels": pv}
+
+        # ---- the step with a shared reweighting network as the meta learner (Sec. 4.1): same sweeps and forward,
+        # plus the reduction of the per-sample differences to the network's gradient ----
+        if with_e2e and not flat and not args.no_variants:
+            hidden = 100
+            lam_r = (0.5 * torch.randn(3 * hidden + 1, generator=torch.Generator().manual_seed(0))).to(dev)
+            mg_r = torch.empty(3 * hidden + 1, dtype=torch.float32, device=dev)
+
+            def rw_step():
+                S.sama_step_reweight(ctx, mlp, n, d["theta"], d["m"], d["s"], d["g_base"], d["g_meta"], adam, alpha,
+                                     d["X"], d["y"], B, hidden, lam_r, p, tp, tm, mg_r, None, None, stream)
+            for _ in range(3):
+                rw_step()
+            Kr = min(total_steps, 100)
+            evr = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(Kr)]
+            for a_, b_ in evr:
+                flush_buf.fill_(1)
+                a_.record(stream)
+                rw_step()
+                b_.record(stream)
+            torch.cuda.synchronize()
+            msr = sum(a_.elapsed_time(b_) for a_, b_ in evr) / Kr
+            out["shared_reweighting_network"] = {"hidden": hidden, "dim_lambda": 3 * hidden + 1, "ms_per_step": msr,
+                                                 "value": group.world * 1e3 / group.max_over_ranks(msr, dev),
+                                                 "unit": "steps/s", "steps": Kr}
 
         # ---- end to end through the host-buffer entry point ----
         if with_e2e and not flat and not args.no_e2e:
@@ -510,6 +535,73 @@ class Bench:
     store_theta_pm = True   # the benchmark asks sama_step for theta+ and theta- (the paper's nudge uses theta-)
 
 
+def biased_regression_stage(b, seed):
+    """Appendix E's study with the meta gradient computed by the library: 100 meta updates at beta = 0.1 on the
+    small workload (base level solved in closed form here, with numpy; plain gradient descent on lambda with step
+    1 / lambda_max of the update's linear map), reporting cos(g_true, g_SAMA) and ||lambda_t - lambda*||; and the
+    time of one SAMA meta-gradient step (direct gradient, adaptation, perturbation, central difference) on
+    both sizes.  The figure in the paper prints no numbers, so there is nothing to compare the values with."""
+    torch, S, dev, stream = b.torch, b.S, b.dev, b.stream
+    out = {}
+    for name, cfg in W.BIASREG.items():
+        w = W.biased_regression(cfg, seed)
+        d, nv = cfg.d, cfg.n_val
+        ctx = S.sama_create(b.local, d, 0, None)
+        t = {k: torch.from_numpy(np.ascontiguousarray(w[k])).to(dev) for k in ("Xv", "yv")}
+        fl = lambda: torch.empty(d, dtype=torch.float32, device=dev)
+        g, p, wp, wm, mg = fl(), fl(), fl(), fl(), fl()
+        w_dev, lam_dev = fl(), fl()
+        sgd = S.Adam(identity=True)
+
+        def step():
+            S.sama_biasreg_step(ctx, d, nv, t["Xv"], t["yv"], w_dev, lam_dev, cfg.beta, None, None, None, sgd, 1.0,
+                                g, p, wp, wm, mg, stream)
+        rec = {"d": d, "n": cfg.n, "n_val": nv, "beta": cfg.beta}
+        if d <= 512:
+            X, y, Xv, yv = (w[k].astype(np.float64) for k in ("X", "y", "Xv", "yv"))
+            H = X.T @ X + cfg.beta * np.eye(d)
+            Hi = np.linalg.inv(H)
+            A = cfg.beta * Xv @ Hi
+            lam_star = np.linalg.solve(A.T @ A, A.T @ (yv - Xv @ (Hi @ (X.T @ y))))
+            eta = 1.0 / np.linalg.eigvals(4 * cfg.beta ** 2 * (Xv.T @ Xv) @ Hi).real.max()
+            lam = w["lam0"].astype(np.float64)
+            cosv, dist = [], []
+            for _ in range(cfg.meta_updates):
+                w_star = Hi @ (X.T @ y + cfg.beta * lam)
+                w_dev.copy_(torch.from_numpy(w_star.astype(np.float32)))
+                lam_dev.copy_(torch.from_numpy(lam.astype(np.float32)))
+                step()
+                torch.cuda.synchronize()
+                gs = mg.cpu().numpy().astype(np.float64)
+                gt = 2 * cfg.beta * (Hi @ (Xv.T @ (Xv @ w_star - yv)))
+                cosv.append(float(gs @ gt / (np.linalg.norm(gs) * np.linalg.norm(gt))))
+                dist.append(float(np.linalg.norm(lam - lam_star)))
+                lam = lam - eta * gs
+            rec["study"] = {"meta_updates": cfg.meta_updates, "cos_first": cosv[0], "cos_min": min(cosv),
+                            "cos_last": cosv[-1], "dist_first": dist[0], "dist_last": dist[-1],
+                            "dist_monotone": all(y_ < x_ for x_, y_ in zip(dist, dist[1:]))}
+        else:
+            w_dev.copy_(torch.from_numpy(w["w_true"]))
+            lam_dev.copy_(torch.from_numpy(w["lam0"]))
+        for _ in range(5):
+            step()
+        K = 50
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        for a_, b_ in ev:
+            b.flush_buf.fill_(1)
+            a_.record(stream)
+            step()
+            b_.record(stream)
+        torch.cuda.synchronize()
+        ms = sum(a_.elapsed_time(b_) for a_, b_ in ev) / K
+        rec["ms_per_meta_gradient"] = ms
+        rec["direct_grad_gbs"] = 4.0 * d * nv / (ms * 1e-3) / 1e9   # X' read once: the step's algorithmic bytes
+        rec["device_status"] = int(S.sama_device_status(ctx))
+        S.sama_destroy(ctx)
+        out[name] = rec
+    return out
+
+
 def brief(r):
     """What the line keeps of a secondary workload."""
     keep = {k: r[k] for k in ("value", "unit", "ms_per_step", "inner_reps", "timed_steps", "clocks", "forward_path",
@@ -530,6 +622,8 @@ def main():
     ap.add_argument("--gemm-mode", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-variants", action="store_true",
+                    help="skip the extra passes on the headline workload (theta+ not stored; shared reweighting network)")
     ap.add_argument("--no-extras", action="store_true",
                     help="time only --workload (the other workloads are added by default on one GPU)")
     ap.add_argument("--region-s", type=float, default=1.2, help="target length of the primary timed region")
@@ -557,7 +651,7 @@ def main():
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic"}
     for k in ("inner_reps", "timed_steps", "config", "clocks", "gpu_launches", "device_status", "forward_path",
               "wall_s_timed_region", "roofline", "rooflines", "kernels", "meta_grad", "e2e", "adapt_perturb_gbs",
-              "without_theta_plus_output"):
+              "without_theta_plus_output", "shared_reweighting_network"):
         if k in r:
             out[k] = r[k]
 
@@ -583,6 +677,7 @@ def main():
             extras[ex] = brief(b.measure(ex, wx, 0.6))
             del wx
         out["workloads"] = extras
+        out["biased_regression"] = biased_regression_stage(b, seed)
         # the metric's three parts in one place
         out["summary"] = {
             "steps_per_s": dict([(PRIMARY, r["value"])] + [(k, v["value"]) for k, v in extras.items()

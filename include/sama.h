@@ -271,6 +271,14 @@ float* sama_ctx_loss_diff(sama_ctx* ctx);
  * the last call in *status_out and clears them. */
 int sama_device_status(sama_ctx* ctx, void* stream, int32_t* status_out);
 
+/* Self-test of the bounded waits.  Every wait inside the tensor-core kernels (on a copy, on a peer CTA, on an
+ * arrival counter) gives up after a cycle limit, raises SAMA_DEV_TIMEOUT and lets the kernel return.  This
+ * launches one warp that waits, with that same routine, on a barrier nothing ever arrives on, for at most
+ * limit_cycles (1 .. 2e9) SM clock cycles.  Afterwards sama_device_status reports SAMA_DEV_TIMEOUT, the context
+ * and the device remain usable, and *waited_cycles_out (one int64 on the device, or NULL) holds how long the
+ * wait lasted.  Nothing faults, traps or spins without bound. */
+int sama_selftest_wait_expiry(sama_ctx* ctx, int64_t limit_cycles, int64_t* waited_cycles_out, void* stream);
+
 /* cudaError_t value of the last failed runtime call on this context (0 if none). */
 int sama_last_cuda_error(sama_ctx* ctx);
 

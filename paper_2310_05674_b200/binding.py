@@ -111,6 +111,7 @@ lib.sama_ctx_sumsq.restype = _vp
 lib.sama_ctx_eps_fd.argtypes = [_vp]
 lib.sama_ctx_eps_fd.restype = _vp
 lib.sama_device_status.argtypes = [_vp, _vp, C.POINTER(C.c_int32)]
+lib.sama_selftest_wait_expiry.argtypes = [_vp, C.c_int64, _vp, _vp]
 lib.sama_last_cuda_error.argtypes = [_vp]
 lib.sama_mlp_param_count.argtypes = [C.POINTER(sama_mlp_t)]
 lib.sama_mlp_param_count.restype = C.c_int64
@@ -277,6 +278,11 @@ def sama_device_status(ctx, stream=None) -> int:
     out = C.c_int32(0)
     _check(lib.sama_device_status(ctx, _stream(stream), C.byref(out)), "sama_device_status")
     return out.value
+
+
+def sama_selftest_wait_expiry(ctx, limit_cycles, waited_cycles_out=None, stream=None) -> int:
+    return _check(lib.sama_selftest_wait_expiry(ctx, int(limit_cycles), _ptr(waited_cycles_out), _stream(stream)),
+                  "sama_selftest_wait_expiry")
 
 
 def sama_last_cuda_error(ctx) -> int:

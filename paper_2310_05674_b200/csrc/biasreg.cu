@@ -9,8 +9,8 @@
 //
 // The direct gradient reads X' once from HBM: a block takes a contiguous run of rows, eight at a time; each warp
 // forms one residual r_i = x_i . w - y_i, then all threads add r_i x_i into the block's partial gradient in
-// shared memory (the rows come back from L1 / L2).  Blocks are added in block order by the last block to
-// arrive.  Accumulation is double throughout; nothing depends on scheduling.
+// shared memory (the rows come back from L1 / L2).  A second small kernel adds the blocks' partials column by
+// column in block order.  Accumulation is double throughout; nothing depends on scheduling.
 #include "sama_internal.h"
 
 namespace sama {
@@ -21,36 +21,46 @@ constexpr int kThreads = 256;
 constexpr int kRows = kThreads / 32;  // rows in flight per block = warps
 
 __global__ void __launch_bounds__(kThreads)
-biasreg_direct_grad_kernel(int d, int n_val, const float* __restrict__ Xv, const float* __restrict__ yv,
-                           const float* __restrict__ w, float* __restrict__ g_out, float* __restrict__ loss_out,
-                           double* partials, DeviceScalars* sc) {
+biasreg_partials_kernel(int d, int n_val, const float* __restrict__ Xv, const float* __restrict__ yv,
+                        const float* __restrict__ w, double* __restrict__ partials) {
     extern __shared__ double g_s[];        // [d] partial gradient, then [kRows] residuals
     double* r_s = g_s + d;
-    __shared__ bool is_last;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int c = threadIdx.x; c < d; c += kThreads) g_s[c] = 0.0;
     // this block's rows: a contiguous run, the same for every launch of this shape
     const int per = (n_val + gridDim.x - 1) / gridDim.x;
     const int row0 = blockIdx.x * per, row1 = min(n_val, row0 + per);
-    double sq = 0.0;                        // sum of r_i^2 over this block's rows (thread 0 of each warp)
+    double sq = 0.0;                        // sum of r_i^2 over this warp's rows (lane 0)
     __syncthreads();
     for (int base = row0; base < row1; base += kRows) {
         const int i = base + warp;
         double r = 0.0;
         if (i < row1) {
             const float* x = Xv + (int64_t)i * d;
-            for (int c = lane; c < d; c += 32) r = fma((double)x[c], (double)w[c], r);
+            double r0 = 0.0, r1 = 0.0, r2 = 0.0, r3 = 0.0;   // four independent chains: eight loads in flight
+            int c = lane;
+            for (; c + 96 < d; c += 128) {
+                r0 = fma((double)x[c], (double)w[c], r0);
+                r1 = fma((double)x[c + 32], (double)w[c + 32], r1);
+                r2 = fma((double)x[c + 64], (double)w[c + 64], r2);
+                r3 = fma((double)x[c + 96], (double)w[c + 96], r3);
+            }
+            for (; c < d; c += 32) r0 = fma((double)x[c], (double)w[c], r0);
+            r = (r0 + r1) + (r2 + r3);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) r += __shfl_xor_sync(0xffffffffu, r, o);
             r -= (double)yv[i];
             if (lane == 0) sq += r * r;
         }
-        if (lane == 0) r_s[warp] = (i < row1) ? r : 0.0;
+        if (lane == 0) r_s[warp] = (i < row1) ? r : 0.0;   // a row past the end contributes nothing
         __syncthreads();
-        const int rows = min(kRows, row1 - base);
         for (int c = threadIdx.x; c < d; c += kThreads) {
+            float xv[kRows];
+#pragma unroll
+            for (int k = 0; k < kRows; ++k) xv[k] = (base + k < row1) ? Xv[(int64_t)(base + k) * d + c] : 0.f;
             double a = g_s[c];
-            for (int k = 0; k < rows; ++k) a = fma((double)Xv[(int64_t)(base + k) * d + c], r_s[k], a);
+#pragma unroll
+            for (int k = 0; k < kRows; ++k) a = fma((double)xv[k], r_s[k], a);
             g_s[c] = a;
         }
         __syncthreads();
@@ -65,22 +75,21 @@ biasreg_direct_grad_kernel(int d, int n_val, const float* __restrict__ Xv, const
         for (int k = 0; k < kRows; ++k) t += r_s[k];
         mine[d] = t;
     }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const unsigned prev = atomicAdd(&sc->counter, 1u);
-        is_last = (prev == gridDim.x - 1);
-    }
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-    for (int c = threadIdx.x; c <= d; c += kThreads) {
-        double t = 0.0;
-        for (unsigned b = 0; b < gridDim.x; ++b) t += __ldcg(partials + (size_t)b * (d + 1) + c);
-        if (c < d) g_out[c] = (float)(2.0 * t);
-        else if (loss_out) *loss_out = (float)t;
-    }
-    if (threadIdx.x == 0) sc->counter = 0u;
+}
+
+// Column c of the result = 2 x (sum over blocks, in block order, of their partials); column d is the meta loss.
+__global__ void __launch_bounds__(128)
+biasreg_reduce_kernel(int d, int blocks, const double* __restrict__ partials, float* __restrict__ g_out,
+                      float* __restrict__ loss_out) {
+    pdl_trigger();
+    pdl_wait();
+    const int c = blockIdx.x * 128 + threadIdx.x;
+    if (c > d) return;
+    double t = 0.0;
+#pragma unroll 8
+    for (int b = 0; b < blocks; ++b) t += __ldcg(partials + (size_t)b * (d + 1) + c);
+    if (c < d) g_out[c] = (float)(2.0 * t);
+    else if (loss_out) *loss_out = (float)t;
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -106,7 +115,7 @@ biasreg_fd_kernel(int64_t d, const float* __restrict__ w_plus, const float* __re
 
 int biasreg_grid(const sama_ctx* ctx, int n_val) {
     int g = (n_val + kRows - 1) / kRows;
-    if (g > ctx->sm_count) g = ctx->sm_count;
+    if (g > 2 * ctx->sm_count) g = 2 * ctx->sm_count;
     return g < 1 ? 1 : g;
 }
 
@@ -114,14 +123,20 @@ cudaError_t launch_biasreg_direct_grad(sama_ctx* ctx, int d, int n_val, const fl
                                        const float* w, float* g_out, float* loss_out, cudaStream_t st) {
     const size_t smem = sizeof(double) * ((size_t)d + kRows);
     if (smem > 48 * 1024) {
-        const cudaError_t e = cudaFuncSetAttribute(biasreg_direct_grad_kernel,
+        const cudaError_t e = cudaFuncSetAttribute(biasreg_partials_kernel,
                                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
+    const int grid = biasreg_grid(ctx, n_val);
+    {
+        KernelScope scope(ctx, SAMA_K_BIASREG_GRAD, -1, st);
+        biasreg_partials_kernel<<<grid, kThreads, smem, st>>>(d, n_val, Xv, yv, w, ctx->br_partials);
+        const cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
     KernelScope scope(ctx, SAMA_K_BIASREG_GRAD, -1, st);
-    biasreg_direct_grad_kernel<<<biasreg_grid(ctx, n_val), kThreads, smem, st>>>(d, n_val, Xv, yv, w, g_out, loss_out,
-                                                                                 ctx->br_partials, ctx->scalars);
-    return cudaGetLastError();
+    return launch_dependent(biasreg_reduce_kernel, dim3((d + 1 + 127) / 128), dim3(128), 0, st, d, grid,
+                            (const double*)ctx->br_partials, g_out, loss_out);
 }
 
 cudaError_t launch_biasreg_fd(sama_ctx* ctx, int64_t d, const float* w_plus, const float* w_minus,

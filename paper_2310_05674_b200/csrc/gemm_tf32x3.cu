@@ -89,7 +89,8 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait: false if the phase did not complete within kWaitCycles, or if another role of the CTA
 // has given up meanwhile (`abort`, looked at only once the first try has failed).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile uint32_t* abort = nullptr) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile uint32_t* abort = nullptr,
+                                          long long limit = kWaitCycles) {
     if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
@@ -97,7 +98,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const v
         for (int i = 0; i < 256; ++i)
             if (mbar_try(bar, parity)) return true;
         if (abort && *abort) return false;
-        if (clock64() - t0 > kWaitCycles) return false;
+        if (clock64() - t0 > limit) return false;
     }
 }
 
@@ -819,6 +820,27 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     }
 }
 
+// The bounded wait on its own: one warp initialises a barrier on which nothing ever arrives and waits on it with
+// the product kernels' wait routine and a caller-chosen limit.  The wait runs out, the status word gets
+// SAMA_DEV_TIMEOUT, the kernel returns normally.  (How a test exercises the expiry path: no fault, no trap, no
+// unbounded spin.)
+__global__ void __launch_bounds__(32)
+wait_expiry_kernel(long long limit_cycles, int32_t* status, long long* waited_cycles) {
+    __shared__ alignas(8) unsigned long long bar_storage;
+    const uint32_t bar = smem_u32(&bar_storage);
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) {
+        const long long t0 = clock64();
+        const bool completed = mbar_wait(bar, 0, nullptr, limit_cycles);
+        if (!completed) atomicOr(status, (int)SAMA_DEV_TIMEOUT);
+        if (waited_cycles) *waited_cycles = clock64() - t0;
+    }
+}
+
 // Splits rows of a dense fp32 matrix [rows][cols] into TF32 hi / lo with the row
 // length padded to ld_out (zeros).  grid.z selects the branch (source pointer
 // and output slab).
@@ -1040,6 +1062,11 @@ cudaError_t launch_split_tf32(sama_ctx* ctx, const float* src0, const float* src
     const dim3 grid((unsigned)blocks, 1, branches);
     return vec ? launch_dependent(split_tf32_kernel<true>, grid, dim3(256), 0, st, a)
                : launch_dependent(split_tf32_kernel<false>, grid, dim3(256), 0, st, a);
+}
+
+cudaError_t launch_wait_expiry(sama_ctx* ctx, long long limit_cycles, long long* waited_cycles, cudaStream_t st) {
+    wait_expiry_kernel<<<1, 32, 0, st>>>(limit_cycles, &ctx->scalars->status, waited_cycles);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_split_transpose_tf32(sama_ctx* ctx, const float* src, int64_t rows, int cols, float* hi, float* lo,

@@ -681,7 +681,7 @@ int sama_biasreg_direct_grad(sama_ctx* ctx, int32_t d, int32_t n_val, const floa
         cudaFree(ctx->br_partials);
         ctx->br_partials = nullptr;
         ctx->br_partials_doubles = 0;
-        const size_t take = (size_t)ctx->sm_count * ((size_t)d + 1);
+        const size_t take = 2 * (size_t)ctx->sm_count * ((size_t)d + 1);
         if (cudaMalloc(&ctx->br_partials, sizeof(double) * take) != cudaSuccess) { cudaGetLastError(); return SAMA_ERR_NOMEM; }
         ctx->br_partials_doubles = take;
     }
@@ -824,6 +824,17 @@ int sama_device_status(sama_ctx* ctx, void* stream, int32_t* status_out) {
     SAMA_CUDA(ctx, cudaMemsetAsync(&ctx->scalars->status, 0, 4, st));
     SAMA_CUDA(ctx, cudaStreamSynchronize(st));
     *status_out = v;
+    return SAMA_OK;
+}
+
+int sama_selftest_wait_expiry(sama_ctx* ctx, int64_t limit_cycles, int64_t* waited_cycles_out, void* stream) {
+    if (!ctx) return SAMA_ERR_NULL;
+    if (limit_cycles < 1 || limit_cycles > (int64_t)2000000000) return SAMA_ERR_PARAM;   // at most about a second
+    if (!aligned(waited_cycles_out, 8)) return SAMA_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SAMA_ERR_CUDA;
+    SAMA_CUDA(ctx, launch_wait_expiry(ctx, (long long)limit_cycles, reinterpret_cast<long long*>(waited_cycles_out),
+                                      (cudaStream_t)stream));
     return SAMA_OK;
 }
 

@@ -268,6 +268,7 @@ cudaError_t launch_split_transpose_tf32(sama_ctx* ctx, const float* src, int64_t
 cudaError_t launch_split_tf32(sama_ctx* ctx, const float* src0, const float* src1, int branches, int64_t rows,
                               int cols, float* hi, float* lo, int64_t slab, cudaStream_t st);
 cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st);
+cudaError_t launch_wait_expiry(sama_ctx* ctx, long long limit_cycles, long long* waited_cycles, cudaStream_t st);
 cudaError_t tc_state_create(sama_ctx* ctx);  // with ctx->device current and ctx->sm_count set
 void tc_state_destroy(sama_ctx* ctx);
 

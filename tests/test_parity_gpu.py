@@ -555,3 +555,27 @@ def test_argument_errors_are_caught_on_the_host():
     # a context without a model cannot run the forward pass
     with Ctx(n) as ctx:
         assert status(B.sama_fd_metagrad, ctx.h, B.MLP((8, 4, 3)), a[0], a[1], X, y, lam, 5, eps, mg) == B.SAMA_ERR_SIZE
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_not_hung():
+    """The expiry path of the kernels' bounded waits, exercised without any fault: a wait on a barrier nothing
+    arrives on, limited to about a millisecond, ends by itself, raises SAMA_DEV_TIMEOUT in the status word, and
+    leaves the context and the device usable (a step right after gives the usual result)."""
+    cfg = W.CONFIGS["tiny"]
+    w = W.mlp_workload(cfg, 0)
+    with Ctx(cfg.n_params, cfg.batch, cfg.dims) as ctx:
+        before = run_step(ctx, cfg, w, B.Adam(), 1e-2)
+        waited = torch.zeros(1, dtype=torch.int64, device=DEV)
+        limit = 2_000_000                       # ~1 ms at 2 GHz
+        B.sama_selftest_wait_expiry(ctx.h, limit, waited)
+        assert B.sama_device_status(ctx.h) == B.SAMA_DEV_TIMEOUT
+        assert limit < int(waited.item()) < 50 * limit
+        assert B.sama_device_status(ctx.h) == 0          # reading cleared it
+        after = run_step(ctx, cfg, w, B.Adam(), 1e-2)
+        assert after["status"] == 0 and np.array_equal(after["metagrad"], before["metagrad"])
+        with pytest.raises(B.SamaError) as e:
+            B.sama_selftest_wait_expiry(ctx.h, 0)
+        assert e.value.status == B.SAMA_ERR_PARAM
+        with pytest.raises(B.SamaError) as e:
+            B.sama_selftest_wait_expiry(ctx.h, 10 ** 12)
+        assert e.value.status == B.SAMA_ERR_PARAM
