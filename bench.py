@@ -282,7 +282,9 @@ class Bench:
         mg = torch.empty(max(B, 1), dtype=torch.float32, device=dev)
         flush_buf = self.flush_buf
 
-        outputs = {"plus": tp, "minus": tm}
+        outputs = {"plus": tp if args.theta_outputs == "both" else None,
+                   "minus": tm if args.theta_outputs != "none" else None}
+        self.store_theta_pm = args.theta_outputs == "both"
 
         def one_step():
             if flat:
@@ -389,7 +391,8 @@ class Bench:
             # the perturbation of Sec. 3.2 is 16 B/element (theta, p in; theta+, theta- out); what the same sweep
             # also writes for the tensor-core forward (hi / lo of W+-: 32 B/element unless theta+- are not
             # stored, and the split of X) is operand preparation, reported beside it
-            moved = (40.0 if self.store_theta_pm else 32.0) * n + (12.0 * B * cfg.dims[0] if cfg else 0.0)
+            stored = {"both": 8.0, "minus": 4.0, "none": 0.0}[args.theta_outputs]
+            moved = (32.0 + stored) * n + (12.0 * B * cfg.dims[0] if cfg else 0.0)
             rooflines["perturb_split"] = hbm_roof("perturb_split", 16.0 * n, moved=moved)
         if "fused_sweep" in per_kernel:   # adaptation + norm + perturbation (+ operand split) in one launch
             moved = (44.0 if self.store_theta_pm else 36.0) * n + 16.0 * n + (12.0 * B * cfg.dims[0] if cfg else 0.0)
@@ -450,7 +453,7 @@ class Bench:
                 key = S.KERNEL_KINDS.get(kind, str(kind))
                 pv[key] = pv.get(key, 0.0) + t / min(Kv, 20)
             S.sama_profile_enable(ctx, 0)
-            outputs["plus"] = tp
+            outputs["plus"] = tp if args.theta_outputs == "both" else None
             out["without_theta_plus_output"] = {"value": group.world * 1e3 / group.max_over_ranks(msv, dev), "unit": "steps/s",
                                                 "ms_per_step": msv, "steps": Kv, "kernels": pv}
 
@@ -622,6 +625,9 @@ def main():
     ap.add_argument("--gemm-mode", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--theta-outputs", default="both", choices=["both", "minus", "none"],
+                    help="which of theta+ / theta- the timed step asks sama_step to store (default both; the "
+                         "forward needs neither)")
     ap.add_argument("--no-variants", action="store_true",
                     help="skip the extra passes on the headline workload (theta+ not stored; shared reweighting network)")
     ap.add_argument("--no-extras", action="store_true",

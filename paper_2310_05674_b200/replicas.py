@@ -60,6 +60,17 @@ class Replicas:
             t /= self.world
         return t
 
+    def shard_range(self, n: int, align: int = 4):
+        """This rank's contiguous share [lo, hi) of a flat vector of n elements, boundaries at multiples of
+        ``align`` (16-byte groups for fp32), the remainder going to the last rank.  For running adaptation and
+        perturbation on a sharded parameter vector: every rank calls sama_adapt on its share, the ranks'
+        sums of squares are added with all_reduce_sum (one double: the norm of Sec. 3.2 is global), and
+        sama_perturb takes that sum as its p_sumsq argument."""
+        per = (n // self.world) // align * align
+        lo = self.rank * per
+        hi = n if self.rank == self.world - 1 else lo + per
+        return lo, hi
+
     def aggregate_rate(self, units_per_rank: float, seconds_this_rank: float, device: str = "cpu") -> float:
         """Whole-job throughput: all ranks' units over the slowest rank's time."""
         return self.world * units_per_rank / self.max_over_ranks(seconds_this_rank, device)

@@ -142,6 +142,29 @@ def test_zero_state_value_of_the_printed_approximation():
             assert Jp + Jm == pytest.approx(0.0, abs=1e-6 * max(abs(lim), 1e-12))
 
 
+def test_other_optimisers_are_arguments_of_the_same_matrix():
+    """Appendix C's last sentence (other optimisers' matrices "can be similarly derived"), checked by differentiating
+    their updates numerically.  RMSprop, u = lr g / (sqrt(b s + (1-b) g^2) + eps), is the Adam matrix with beta1 = 0
+    and no bias correction.  SGD with momentum, u = lr (mu buf + g), has du/dg = lr: a multiple of the identity,
+    which the norm-scaled step of Sec. 3.2 cannot tell from identity = 1 (same theta+-, same direction)."""
+    rng = np.random.default_rng(7)
+    for _ in range(300):
+        b, lr, eps = float(rng.uniform(0.8, 0.999)), float(10 ** rng.uniform(-4, -2)), float(10 ** rng.uniform(-10, -6))
+        s, g = np.float32(abs(rng.normal()) * 1e-5 + 1e-8), np.float32(rng.normal() * 3e-3)
+        u = lambda x: LD(lr) * x / (np.sqrt(LD(b) * LD(s) + (1 - LD(b)) * x * x) + LD(eps))
+        h = LD(1e-4) * max(abs(LD(g)), np.sqrt(LD(s)))
+        d = (-u(LD(g) + 2 * h) + 8 * u(LD(g) + h) - 8 * u(LD(g) - h) + u(LD(g) - 2 * h)) / (12 * h)
+        J = jac(0.123, s, g, oracle.Adam(lr, 0.0, b, eps, 1, bias_correction=False))
+        assert J == pytest.approx(float(d), rel=1e-6)
+    w = W.flat_vector(500, 8)
+    lr, mu = 0.05, 0.9
+    p_sgd = lr * w["g_meta"].astype(np.float64)                 # (d/dg)[lr (mu buf + g)] * g_meta
+    tp_a, tm_a, _, _ = oracle.perturb(w["theta"], p_sgd, 1e-2)
+    tp_b, tm_b, _, _ = oracle.perturb(w["theta"], oracle.adapt(w["m"], w["s"], None, w["g_meta"], oracle.Adam(identity=True)), 1e-2)
+    np.testing.assert_allclose(tp_a, tp_b, rtol=0, atol=1e-15)
+    np.testing.assert_allclose(tm_a, tm_b, rtol=0, atol=1e-15)
+
+
 def test_identity_mode_is_bit_exact_and_sgd_reduction():
     w = W.adam_state(1000, 3)
     p = oracle.adapt(w["m"], w["s"], w["g_base"], w["g_meta"], oracle.Adam(identity=True))

@@ -34,6 +34,7 @@ ADAMS = {
     "dropeps": B.Adam(drop_eps_term=True),
     "identity": B.Adam(identity=True),
     "odd": B.Adam(lr=3e-2, beta1=0.8, beta2=0.99, eps=1e-6, step=7),
+    "rmsprop": B.Adam(lr=1e-2, beta1=0.0, beta2=0.99, eps=1e-8, bias_correction=False),   # RMSprop's matrix (Appendix C, last sentence)
 }
 
 

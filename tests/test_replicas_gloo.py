@@ -121,3 +121,57 @@ def test_one_gradient_synchronisation_gives_the_batch_meta_gradient(tmp_path):
         assert p.returncode == 0, err[-2000:]
         d = json.loads([l for l in out.splitlines() if l.startswith("RESULT ")][0][7:])
         assert d["err"] < 1e-10 and d["mean_err"] < 1e-10 and d["local_differs"]
+
+
+CHILD_SHARD = textwrap.dedent("""
+    import json, sys
+    sys.path.insert(0, %r)
+    import numpy as np, torch
+    import oracle
+    from paper_2310_05674_b200 import replicas, workloads as W
+    r = replicas.init(backend="gloo")
+    n, alpha = 100003, 0.37
+    w = W.flat_vector(n, 5)                               # the same vector on both ranks; each takes its share
+    adam = oracle.Adam(step=7)
+    lo, hi = r.shard_range(n)
+    p = oracle.adapt(w["m"][lo:hi], w["s"][lo:hi], w["g_base"][lo:hi], w["g_meta"][lo:hi], adam)
+    ss = torch.tensor([oracle.sumsq(p)], dtype=torch.float64)
+    r.all_reduce_sum(ss)                                  # the one exchange: 8 bytes
+    tp, tm, eps, bad = oracle.perturb_given_sumsq(w["theta"][lo:hi], p, float(ss.item()), alpha)
+    p_all = oracle.adapt(w["m"], w["s"], w["g_base"], w["g_meta"], adam)
+    tp_all, tm_all, eps_all, _ = oracle.perturb(w["theta"], p_all, alpha)
+    out = {"rank": r.rank, "lo": lo, "hi": hi, "bad": bool(bad),
+           "eps_rel": abs(eps - eps_all) / eps_all,
+           "same": bool(np.array_equal(p, p_all[lo:hi])),
+           "tp_err": float(np.abs(tp - tp_all[lo:hi]).max()), "tm_err": float(np.abs(tm - tm_all[lo:hi]).max())}
+    r.barrier()
+    r.close()
+    print("RESULT " + json.dumps(out), flush=True)
+""") % ROOT
+
+
+def test_sharded_vector_needs_one_eight_byte_exchange(tmp_path):
+    """Sec. 3.2's norm is over the whole vector: two gloo ranks adapt their contiguous shares, add their sums of
+    squares once, and perturb their shares with the global step size; together that is the unsharded result."""
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    script = tmp_path / "child_shard.py"
+    script.write_text(CHILD_SHARD)
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE="2",
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env, stdout=subprocess.PIPE,
+                                      stderr=subprocess.PIPE, text=True))
+    import json
+    res = {}
+    for p in procs:
+        out, err = p.communicate(timeout=180)
+        assert p.returncode == 0, err[-2000:]
+        d = json.loads([l for l in out.splitlines() if l.startswith("RESULT ")][0][7:])
+        res[d["rank"]] = d
+    assert res[0]["lo"] == 0 and res[0]["hi"] == res[1]["lo"] and res[1]["hi"] == 100003 and res[0]["hi"] % 4 == 0
+    for d in res.values():
+        assert d["same"] and not d["bad"] and d["eps_rel"] < 1e-12 and d["tp_err"] < 1e-12 and d["tm_err"] < 1e-12
