@@ -584,10 +584,22 @@ int sama_step(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* thet
         xjob.cols = mlp->dims[0];
         xjob.ld_out = (mlp->dims[0] + 31) & ~31;
     }
+    bool swept = false;
     if (one_launch) {
-        SAMA_CUDA(ctx, launch_fused_sweep(ctx, n, theta, m, s, c.identity ? nullptr : g_base, g_meta, c, alpha, p_out,
-                                          theta_plus, theta_minus, lay, ctx->w_split, ctx->w_split + ctx->w_split_half,
-                                          ctx->pm_small, xjob, st));
+        const cudaError_t e = launch_fused_sweep(ctx, n, theta, m, s, c.identity ? nullptr : g_base, g_meta, c, alpha,
+                                                 p_out, theta_plus, theta_minus, lay, ctx->w_split,
+                                                 ctx->w_split + ctx->w_split_half, ctx->pm_small, xjob, st);
+        if (e == cudaSuccess) {
+            swept = true;
+        } else {
+            // a cooperative launch the device would not take (its blocks must all be resident): nothing has run;
+            // remember that, and take the two launches from here on
+            cudaGetLastError();
+            ctx->fused_sweep_blocks = -1;
+            SAMA_CUDA(ctx, launch_adapt_sumsq(ctx, n, m, s, c.identity ? nullptr : g_base, g_meta, c, p_out, nullptr, st));
+        }
+    }
+    if (swept) {
     } else if (fused) {
         SAMA_CUDA(ctx, launch_perturb_split(ctx, n, theta, p_out, &ctx->scalars->sumsq, alpha, theta_plus,
                                             theta_minus, nullptr, lay, ctx->w_split,
