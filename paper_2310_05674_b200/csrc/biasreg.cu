@@ -20,6 +20,8 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kRows = kThreads / 32;  // rows in flight per block = warps
 
+// VEC: d % 4 == 0 and 16-byte aligned X', w: 16-byte loads, four times as many bytes in flight per thread.
+template <bool VEC>
 __global__ void __launch_bounds__(kThreads)
 biasreg_partials_kernel(int d, int n_val, const float* __restrict__ Xv, const float* __restrict__ yv,
                         const float* __restrict__ w, double* __restrict__ partials) {
@@ -37,15 +39,39 @@ biasreg_partials_kernel(int d, int n_val, const float* __restrict__ Xv, const fl
         double r = 0.0;
         if (i < row1) {
             const float* x = Xv + (int64_t)i * d;
-            double r0 = 0.0, r1 = 0.0, r2 = 0.0, r3 = 0.0;   // four independent chains: eight loads in flight
-            int c = lane;
-            for (; c + 96 < d; c += 128) {
-                r0 = fma((double)x[c], (double)w[c], r0);
-                r1 = fma((double)x[c + 32], (double)w[c + 32], r1);
-                r2 = fma((double)x[c + 64], (double)w[c + 64], r2);
-                r3 = fma((double)x[c + 96], (double)w[c + 96], r3);
+            double r0 = 0.0, r1 = 0.0, r2 = 0.0, r3 = 0.0;   // four independent chains
+            if (VEC) {
+                const float4* x4 = reinterpret_cast<const float4*>(x);
+                const float4* w4 = reinterpret_cast<const float4*>(w);
+                const int q = d >> 2;
+                int c = lane;
+                for (; c + 96 < q; c += 128) {
+                    const float4 a0 = __ldg(x4 + c), a1 = __ldg(x4 + c + 32), a2 = __ldg(x4 + c + 64), a3 = __ldg(x4 + c + 96);
+                    const float4 b0 = __ldg(w4 + c), b1 = __ldg(w4 + c + 32), b2 = __ldg(w4 + c + 64), b3 = __ldg(w4 + c + 96);
+                    r0 = fma((double)a0.x, (double)b0.x, r0); r0 = fma((double)a0.y, (double)b0.y, r0);
+                    r0 = fma((double)a0.z, (double)b0.z, r0); r0 = fma((double)a0.w, (double)b0.w, r0);
+                    r1 = fma((double)a1.x, (double)b1.x, r1); r1 = fma((double)a1.y, (double)b1.y, r1);
+                    r1 = fma((double)a1.z, (double)b1.z, r1); r1 = fma((double)a1.w, (double)b1.w, r1);
+                    r2 = fma((double)a2.x, (double)b2.x, r2); r2 = fma((double)a2.y, (double)b2.y, r2);
+                    r2 = fma((double)a2.z, (double)b2.z, r2); r2 = fma((double)a2.w, (double)b2.w, r2);
+                    r3 = fma((double)a3.x, (double)b3.x, r3); r3 = fma((double)a3.y, (double)b3.y, r3);
+                    r3 = fma((double)a3.z, (double)b3.z, r3); r3 = fma((double)a3.w, (double)b3.w, r3);
+                }
+                for (; c < q; c += 32) {
+                    const float4 a0 = __ldg(x4 + c), b0 = __ldg(w4 + c);
+                    r0 = fma((double)a0.x, (double)b0.x, r0); r0 = fma((double)a0.y, (double)b0.y, r0);
+                    r0 = fma((double)a0.z, (double)b0.z, r0); r0 = fma((double)a0.w, (double)b0.w, r0);
+                }
+            } else {
+                int c = lane;
+                for (; c + 96 < d; c += 128) {
+                    r0 = fma((double)x[c], (double)w[c], r0);
+                    r1 = fma((double)x[c + 32], (double)w[c + 32], r1);
+                    r2 = fma((double)x[c + 64], (double)w[c + 64], r2);
+                    r3 = fma((double)x[c + 96], (double)w[c + 96], r3);
+                }
+                for (; c < d; c += 32) r0 = fma((double)x[c], (double)w[c], r0);
             }
-            for (; c < d; c += 32) r0 = fma((double)x[c], (double)w[c], r0);
             r = (r0 + r1) + (r2 + r3);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) r += __shfl_xor_sync(0xffffffffu, r, o);
@@ -54,14 +80,32 @@ biasreg_partials_kernel(int d, int n_val, const float* __restrict__ Xv, const fl
         }
         if (lane == 0) r_s[warp] = (i < row1) ? r : 0.0;   // a row past the end contributes nothing
         __syncthreads();
-        for (int c = threadIdx.x; c < d; c += kThreads) {
-            float xv[kRows];
+        if (VEC) {
+            const int q = d >> 2;
+            for (int c = threadIdx.x; c < q; c += kThreads) {
+                float4 xv[kRows];
 #pragma unroll
-            for (int k = 0; k < kRows; ++k) xv[k] = (base + k < row1) ? Xv[(int64_t)(base + k) * d + c] : 0.f;
-            double a = g_s[c];
+                for (int k = 0; k < kRows; ++k)
+                    xv[k] = (base + k < row1) ? __ldg(reinterpret_cast<const float4*>(Xv + (int64_t)(base + k) * d) + c)
+                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+                double a0 = g_s[4 * c], a1 = g_s[4 * c + 1], a2 = g_s[4 * c + 2], a3 = g_s[4 * c + 3];
 #pragma unroll
-            for (int k = 0; k < kRows; ++k) a = fma((double)xv[k], r_s[k], a);
-            g_s[c] = a;
+                for (int k = 0; k < kRows; ++k) {
+                    a0 = fma((double)xv[k].x, r_s[k], a0); a1 = fma((double)xv[k].y, r_s[k], a1);
+                    a2 = fma((double)xv[k].z, r_s[k], a2); a3 = fma((double)xv[k].w, r_s[k], a3);
+                }
+                g_s[4 * c] = a0; g_s[4 * c + 1] = a1; g_s[4 * c + 2] = a2; g_s[4 * c + 3] = a3;
+            }
+        } else {
+            for (int c = threadIdx.x; c < d; c += kThreads) {
+                float xv[kRows];
+#pragma unroll
+                for (int k = 0; k < kRows; ++k) xv[k] = (base + k < row1) ? Xv[(int64_t)(base + k) * d + c] : 0.f;
+                double a = g_s[c];
+#pragma unroll
+                for (int k = 0; k < kRows; ++k) a = fma((double)xv[k], r_s[k], a);
+                g_s[c] = a;
+            }
         }
         __syncthreads();
     }
@@ -122,15 +166,20 @@ int biasreg_grid(const sama_ctx* ctx, int n_val) {
 cudaError_t launch_biasreg_direct_grad(sama_ctx* ctx, int d, int n_val, const float* Xv, const float* yv,
                                        const float* w, float* g_out, float* loss_out, cudaStream_t st) {
     const size_t smem = sizeof(double) * ((size_t)d + kRows);
+    const bool vec = (d % 4 == 0) && ((reinterpret_cast<uintptr_t>(Xv) & 15u) == 0) &&
+                     ((reinterpret_cast<uintptr_t>(w) & 15u) == 0);
     if (smem > 48 * 1024) {
-        const cudaError_t e = cudaFuncSetAttribute(biasreg_partials_kernel,
-                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        const cudaError_t e = vec ? cudaFuncSetAttribute(biasreg_partials_kernel<true>,
+                                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                                  : cudaFuncSetAttribute(biasreg_partials_kernel<false>,
+                                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
     const int grid = biasreg_grid(ctx, n_val);
     {
         KernelScope scope(ctx, SAMA_K_BIASREG_GRAD, -1, st);
-        biasreg_partials_kernel<<<grid, kThreads, smem, st>>>(d, n_val, Xv, yv, w, ctx->br_partials);
+        if (vec) biasreg_partials_kernel<true><<<grid, kThreads, smem, st>>>(d, n_val, Xv, yv, w, ctx->br_partials);
+        else biasreg_partials_kernel<false><<<grid, kThreads, smem, st>>>(d, n_val, Xv, yv, w, ctx->br_partials);
         const cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
