@@ -387,16 +387,19 @@ class Bench:
             rooflines["adapt_sumsq"] = hbm_roof("adapt_sumsq", 20.0 * n)
         if "perturb" in per_kernel:
             rooflines["perturb"] = hbm_roof("perturb", 16.0 * n)
+        # Bytes the sweeps move beyond the algorithmic ones: what they also write for the tensor-core forward (hi / lo
+        # of W+-: 32 B/element; none in gemm mode 3, where the product kernel forms them) and the split of X;
+        # theta+- count only where they are stored.
+        stored = {"both": 8.0, "minus": 4.0, "none": 0.0}[args.theta_outputs]
+        prep = 0.0 if args.gemm_mode == 3 else 32.0
+        x_prep = 12.0 * B * cfg.dims[0] if cfg else 0.0
         if "perturb_split" in per_kernel:
-            # the perturbation of Sec. 3.2 is 16 B/element (theta, p in; theta+, theta- out); what the same sweep
-            # also writes for the tensor-core forward (hi / lo of W+-: 32 B/element unless theta+- are not
-            # stored, and the split of X) is operand preparation, reported beside it
-            stored = {"both": 8.0, "minus": 4.0, "none": 0.0}[args.theta_outputs]
-            moved = (32.0 + stored) * n + (12.0 * B * cfg.dims[0] if cfg else 0.0)
-            rooflines["perturb_split"] = hbm_roof("perturb_split", 16.0 * n, moved=moved)
+            # the perturbation of Sec. 3.2 is 16 B/element (theta, p in; theta+, theta- out)
+            read = 8.0 if (prep or stored) else 0.0   # with nothing to store per weight, the weights are not read
+            rooflines["perturb_split"] = hbm_roof("perturb_split", 16.0 * n, moved=(read + stored + prep) * n + x_prep)
         if "fused_sweep" in per_kernel:   # adaptation + norm + perturbation (+ operand split) in one launch
-            moved = (44.0 if self.store_theta_pm else 36.0) * n + 16.0 * n + (12.0 * B * cfg.dims[0] if cfg else 0.0)
-            rooflines["fused_sweep"] = hbm_roof("fused_sweep", 36.0 * n, moved=moved)
+            # reads m, s, g_base, g_meta, theta (p stays in shared memory), writes p
+            rooflines["fused_sweep"] = hbm_roof("fused_sweep", 36.0 * n, moved=(28.0 + stored + prep) * n + x_prep)
         sweep = [k for k in ("adapt_sumsq", "perturb", "perturb_split", "sumsq", "fused_sweep") if k in per_kernel]
         if sweep:   # adaptation + norm + perturbation together: 36 B/element over the sum of their launch times
             t = sum(per_kernel[k]["ms_per_step"] for k in sweep) * 1e-3
@@ -432,7 +435,8 @@ class Bench:
         out = {"value": value, "unit": "steps/s", "ms_per_step": ms_per_step, "steps": args.steps,
                "inner_reps": reps, "timed_steps": total_steps, "config": config_for(name, flat_n),
                "clocks": clocks, "gpu_launches": int(launches), "device_status": int(status),
-               "forward_path": {0: "none", 1: "fp32 FMA", 2: "tensor cores, 3xTF32"}[S.sama_last_forward_path(ctx)],
+               "forward_path": {0: "none", 1: "fp32 FMA", 2: "tensor cores, 3xTF32",
+                                3: "tensor cores, 3xTF32, weights perturbed in the operand stage"}[S.sama_last_forward_path(ctx)],
                "wall_s_timed_region": t_wall, "roofline": roofline, "rooflines": rooflines, "kernels": per_kernel}
         if flat:
             out["adapt_perturb_gbs"] = 36.0 * n / (ms_per_step * 1e-3) / 1e9

@@ -288,14 +288,22 @@ int64_t sama_mlp_param_count(const sama_mlp_t* mlp);
 /* Static text for a sama_status value. */
 const char* sama_status_string(int status);
 
-/* Selects how sama_fd_metagrad (Eq. 5) multiplies matrices: 0 = automatic,
- * 1 = fp32 FMA on the CUDA cores, 2 = tensor cores with each fp32 operand
- * split into two TF32 terms and three products per block (error comparable
- * to fp32).  Returns SAMA_ERR_UNSUPPORTED for a mode this build lacks. */
+/* Selects how the forward pass of Eq. 5 multiplies matrices: 0 = automatic
+ * (the tensor cores where the model fits their workspaces), 1 = fp32 FMA on
+ * the CUDA cores, 2 = tensor cores with each fp32 operand split into two
+ * TF32 terms and three products per block (error comparable to fp32),
+ * 3 = as 2, and in sama_step the product kernel itself forms the weights of
+ * both branches, theta +- eps_fd p (Sec. 3.2), in its operand stage from theta
+ * and p: the perturbed weights then never exist in device memory and the
+ * perturbation sweep writes no operand copy (layers with d_in >= 32, inputs
+ * 16-byte aligned; other layers and the other entry points behave as in 2).
+ * Modes 2 and 3 return SAMA_ERR_SIZE from the forward when the model does
+ * not fit the workspaces.  Returns SAMA_ERR_PARAM for an unknown mode. */
 int sama_set_gemm_mode(sama_ctx* ctx, int mode);
 
 /* How the last forward pass run through this context (sama_fd_metagrad, sama_step, sama_step_host)
- * multiplied matrices: 0 = none yet, 1 = fp32 FMA on the CUDA cores, 2 = tensor cores (3xTF32).  In
+ * multiplied matrices: 0 = none yet, 1 = fp32 FMA on the CUDA cores, 2 = tensor cores (3xTF32), 3 = tensor
+ * cores with the perturbed weights formed in the operand stage (mode 3 of sama_set_gemm_mode).  In
  * automatic mode a model that does not fit the operand workspace sized at sama_create takes path 1,
  * which is several times slower; this query makes that visible. */
 int sama_last_forward_path(sama_ctx* ctx);

@@ -300,6 +300,14 @@ struct SplitDst {
     float* lo;
     float* small;
 };
+// Whether the group of four elements starting at e is a weight of a layer the sweep writes no operands for (so
+// that, when theta+- are not stored either, the group need not even be read).
+__device__ __forceinline__ bool skipped_weight(const SplitLayout& lay, int64_t e) {
+#pragma unroll 1
+    for (int k = 0; k < lay.n_layers; ++k)
+        if (e >= lay.w_off[k] && e < lay.w_off[k] + lay.w_cnt[k]) return ((lay.skip_w >> k) & 1u) != 0;
+    return false;
+}
 __device__ __forceinline__ void emit_split(const SplitLayout& lay, const SplitDst& o, float eps, int64_t i, float4 vt,
                                            float4 vp) {
     float4 a, b;
@@ -327,6 +335,7 @@ __device__ __forceinline__ void emit_split(const SplitLayout& lay, const SplitDs
         *reinterpret_cast<float4*>(small_m + rel64) = b;
         return;
     }
+    if ((lay.skip_w >> l) & 1u) return;   // the product kernel forms this layer's operands itself
     const uint32_t rel = (uint32_t)rel64;
     const uint32_t K = (uint32_t)lay.K[l], Kp = (uint32_t)lay.Kp[l];
     const uint32_t row = rel / K, col = rel - row * K;
@@ -410,6 +419,12 @@ perturb_split_kernel(int64_t n, const float* theta, const float* __restrict__ p,
     auto emit = [&](int64_t i, float4 vt, float4 vp) { emit_split(lay, dst, eps, i, vt, vp); };
 
     int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (!theta_plus && !theta_minus && lay.skip_w != 0u) {
+        // nothing is stored for the skipped layers' weights: only the other groups are read at all
+        for (; i < items; i += stride)
+            if (!skipped_weight(lay, i << 2)) emit(i, ld_stream(t4 + i), ld_stream(p4 + i));
+        i = items;
+    }
     for (; i + stride < items; i += stride * 2) {
         const float4 vt0 = ld_stream(t4 + i), vp0 = ld_stream(p4 + i);
         const float4 vt1 = ld_stream(t4 + i + stride), vp1 = ld_stream(p4 + i + stride);
@@ -533,10 +548,12 @@ fused_sweep_kernel(int64_t n, const float* theta, const float* __restrict__ m, c
         if (bad) atomicOr(&sc->status, (int)SAMA_DEV_DEGENERATE_NORM);
     }
     const SplitDst dst{theta_plus, theta_minus, hi, lo, small};
+    const bool sparse = !theta_plus && !theta_minus && lay.skip_w != 0u;  // most groups have nothing to store
 #pragma unroll 2
     for (int vv = 0; vv < kFusedVec; ++vv) {
         const int64_t i = i0 + stride * vv;
-        if (i < items) emit_split(lay, dst, eps, i, ld_stream(t4 + i), p_s[vv * kThreads + threadIdx.x]);
+        if (i < items && !(sparse && skipped_weight(lay, i << 2)))
+            emit_split(lay, dst, eps, i, ld_stream(t4 + i), p_s[vv * kThreads + threadIdx.x]);
     }
     if (has_tail) emit_split_tail(lay, dst, eps, tail_k, theta[tail_k], tail_p);
 }

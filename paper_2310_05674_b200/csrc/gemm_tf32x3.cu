@@ -28,6 +28,11 @@
 //               after a tile's last chunk it adds the bias, applies ReLU, and stores
 //               fp32 results and / or the next layer's hi/lo operands through a
 //               shared-memory transpose, while the next tile is being multiplied.
+//   warps 2 + EPI .. (XF > 0 only): operand transform.  The weights of the two branches are theta +- eps_fd p
+//               (Sec. 3.2).  Instead of reading them as a pre-split copy, the producer then loads the tile of
+//               theta into the W hi slot and the tile of p into the W lo slot, and these warps replace them in
+//               place by hi / lo of fma(+-eps_fd, p, theta) before the products read them: the perturbed
+//               weights never exist in global memory.
 // A layer with fewer tiles than SMs gives each tile to a cluster of 2 or 4 CTAs that split the
 // contraction and exchange partial sums (see ksplit).
 // Operands are K-major in global memory ([rows][K], K padded to a multiple of
@@ -55,7 +60,8 @@ constexpr int UMMA_K = 8;     // K of one kind::tf32 instruction
 // alternate between two accumulators in tensor memory; the epilogue warps add each finished chunk
 // into fp32 registers (round-to-nearest) while the next chunk is being multiplied.
 constexpr int kChunkKb = 4;
-__host__ __device__ constexpr int threads_for(int epi) { return 64 + 32 * epi; }  // epi = 4 or 8 epilogue warps
+// epi = 4 or 8 epilogue warps, xf = 0 or 2 operand-transform warps
+__host__ __device__ constexpr int threads_for(int epi, int xf = 0) { return 64 + 32 * epi + 32 * xf; }
 constexpr long long kWaitCycles = 4000000000LL;  // ~2 s at 2 GHz
 
 // `wrows` = rows of W one CTA stages per k-block: BN, or BN / 2 when a CTA pair shares the W tile.
@@ -63,6 +69,7 @@ __host__ __device__ constexpr int stage_bytes(int wrows) { return 2 * BM * BKF *
 __host__ __device__ constexpr int stages_for(int wrows) {
     return (200 * 1024) / stage_bytes(wrows) > 5 ? 5 : (200 * 1024) / stage_bytes(wrows);
 }
+constexpr int kXf = 2;  // operand-transform warps of the kernels that form W from theta and p
 constexpr int kStoreStageBytes = 32 * 32 * 4;  // per epilogue warp: a 32 x 32 fp32 block on its way to row-contiguous stores
 __host__ __device__ constexpr int smem_bytes(int wrows) {
     return stages_for(wrows) * stage_bytes(wrows) + 1024 + 256 + 8 * kStoreStageBytes;
@@ -120,6 +127,18 @@ __device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) 
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
+}
+// Bounded wait on a barrier on which another CTA of the cluster arrives with release.cluster.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, const volatile uint32_t* abort) {
+    if (mbar_try_cluster(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_cluster(bar, parity)) return true;
+        if (abort && *abort) return false;
+        if (clock64() - t0 > kWaitCycles) return false;
+    }
 }
 __device__ __forceinline__ void st_cluster_f4(uint32_t addr, float a, float b, float c, float d) {
     asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
@@ -280,7 +299,9 @@ struct TcArgs {
     // tiles, then the `tail_tiles` remaining ones are each shared by two units (half of the k-blocks each).
     int full_rounds, tail_tiles;
     int* flags;            // arrival counters of the shared tail tiles [tail tile][2 halves][2 CTAs], zero between launches
-    uint32_t tx_bytes;     // bytes the four copies of one k-block deliver
+    uint32_t tx_bytes;     // bytes the four copies of one k-block deliver (XF > 0: the two copies of A)
+    uint32_t w_tx_bytes;   // XF > 0: bytes of the theta and p tiles one CTA receives per k-block
+    const float* eps_fd;   // XF > 0: the finite-difference step (device); branch 0 takes +eps_fd, branch 1 -eps_fd
     int32_t* status;
 };
 
@@ -386,8 +407,10 @@ __device__ __forceinline__ void store_block(const TcArgs& args, const float4* st
 // PAIR = true: two CTAs of a cluster work on one 256 x BN tile.  Each stages its own 128 rows of A and half of
 // the W tile; the leader CTA issues cta_group::2 products that read both CTAs' shared memory and write both
 // CTAs' tensor memory.  Per CTA and flop that is fewer operand bytes than two independent 128 x BN tiles.
-template <int BN, bool PAIR, int EPI>
-__global__ void __launch_bounds__(threads_for(EPI), 1)
+// XF > 0: map_w_hi covers this layer's weights inside theta and map_w_lo the same block of p ([N][K] fp32, one
+// slab); XF warps form the operands of theta +- eps_fd p in shared memory.
+template <int BN, bool PAIR, int EPI, int XF>
+__global__ void __launch_bounds__(threads_for(EPI, XF), 1)
 gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
                    const __grid_constant__ CUtensorMap map_w_hi, const __grid_constant__ CUtensorMap map_w_lo,
                    const __grid_constant__ TcArgs args) {
@@ -418,6 +441,11 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
     const uint32_t part_bar = bars + 8u * (2 * STAGES + 4);   // K-split: the other CTAs' partial sums have been written
     const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 5);
     const uint32_t abort_slot = tmem_slot + 4;
+    // XF > 0: theta and p tiles of stage s have landed in this CTA; the W operands of stage s are in place (the
+    // leader's barrier, for a pair)
+    auto wfull_bar = [&](int s) { return bars + 8u * (2 * STAGES + 7 + s); };
+    auto ready_bar = [&](int s) { return bars + 8u * (3 * STAGES + 7 + s); };
+    static_assert(8 * (4 * stages_for(PAIR ? BN / 2 : BN) + 7) <= 256, "barriers fit in front of the store staging");
     volatile uint32_t* abort_flag =
         reinterpret_cast<volatile uint32_t*>(smem_raw + (abort_slot - smem_u32(smem_raw)));
     volatile uint32_t* tmem_ptr_slot =
@@ -484,6 +512,10 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar(s), 1);
             mbar_init(empty_bar(s), 1);
+            if (XF > 0) {
+                mbar_init(wfull_bar(s), 1);
+                mbar_init(ready_bar(s), XF * (PAIR ? 2 : 1));  // one arrival per transform warp (of both CTAs of a pair)
+            }
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(acc_full_bar(b), 1);
@@ -530,29 +562,41 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                     if (issued >= STAGES && !mbar_wait(empty_bar(s), empty_parity, abort_flag)) { raise_timeout(); ok = false; break; }
                     const uint32_t st = base + s * STAGE;
                     const int kx = (kb0 + kb) * BKF;
+                    if (XF > 0) {
+                        // theta into the W hi slot, p into the W lo slot: this CTA's own barrier, for its transform warps
+                        mbar_expect_tx(wfull_bar(s), args.w_tx_bytes);
+                        tma_load_3d(st + 2 * A_BYTES, &map_w_hi, wfull_bar(s), kx, nw0, 0);
+                        tma_load_3d(st + 2 * A_BYTES + W_BYTES, &map_w_lo, wfull_bar(s), kx, nw0, 0);
+                    }
                     if (PAIR) {
                         // both CTAs' copies complete on the leader's barrier, which the leader arms for all of them
                         const uint32_t lbar = full_bar(s) & kPeerBitMask;
                         if (rank == 0) mbar_expect_tx(full_bar(s), args.tx_bytes);
                         tma_load_3d_pair(st, &map_a_hi, lbar, kx, m0, za);
                         tma_load_3d_pair(st + A_BYTES, &map_a_lo, lbar, kx, m0, za);
-                        tma_load_3d_pair(st + 2 * A_BYTES, &map_w_hi, lbar, kx, nw0, br);
-                        tma_load_3d_pair(st + 2 * A_BYTES + W_BYTES, &map_w_lo, lbar, kx, nw0, br);
+                        if (XF == 0) {
+                            tma_load_3d_pair(st + 2 * A_BYTES, &map_w_hi, lbar, kx, nw0, br);
+                            tma_load_3d_pair(st + 2 * A_BYTES + W_BYTES, &map_w_lo, lbar, kx, nw0, br);
+                        }
                     } else {
                         mbar_expect_tx(full_bar(s), args.tx_bytes);
                         tma_load_3d(st, &map_a_hi, full_bar(s), kx, m0, za);
                         tma_load_3d(st + A_BYTES, &map_a_lo, full_bar(s), kx, m0, za);
-                        tma_load_3d(st + 2 * A_BYTES, &map_w_hi, full_bar(s), kx, n0, br);
-                        tma_load_3d(st + 2 * A_BYTES + W_BYTES, &map_w_lo, full_bar(s), kx, n0, br);
+                        if (XF == 0) {
+                            tma_load_3d(st + 2 * A_BYTES, &map_w_hi, full_bar(s), kx, n0, br);
+                            tma_load_3d(st + 2 * A_BYTES + W_BYTES, &map_w_lo, full_bar(s), kx, n0, br);
+                        }
                     }
                     ++issued;
                     if (++s == STAGES) { s = 0; empty_parity ^= 1u; }
                 }
             }
-            if (*abort_flag && rank == 0) {
+            if (*abort_flag) {
                 // let the copies already issued land before the CTA's shared memory goes away
-                for (int i = (issued > STAGES ? issued - STAGES : 0); i < issued; ++i)
-                    mbar_wait(full_bar(i % STAGES), (i / STAGES) & 1);
+                for (int i = (issued > STAGES ? issued - STAGES : 0); i < issued; ++i) {
+                    if (rank == 0) mbar_wait(full_bar(i % STAGES), (i / STAGES) & 1);
+                    if (XF > 0) mbar_wait(wfull_bar(i % STAGES), (i / STAGES) & 1);
+                }
             }
         }
     } else if (warp == 1) {
@@ -573,6 +617,11 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                         if (!mbar_wait(acc_empty_bar(buf), ((chunk >> 1) - 1) & 1, abort_flag)) { raise_timeout(); ok = false; break; }
                     }
                     if (!mbar_wait(full_bar(s), full_parity, abort_flag)) { raise_timeout(); ok = false; break; }
+                    if (XF > 0) {  // the W operands of this stage have been formed (in both CTAs of a pair)
+                        const bool got = PAIR ? mbar_wait_cluster(ready_bar(s), full_parity, abort_flag)
+                                              : mbar_wait(ready_bar(s), full_parity, abort_flag);
+                        if (!got) { raise_timeout(); ok = false; break; }
+                    }
                     tc_fence_after();
                     const uint32_t st = base + s * STAGE;
                     const uint32_t acc = tmem_base + (uint32_t)buf * ACC_COLS;
@@ -606,6 +655,85 @@ gemm_tf32x3_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_co
                     }
                     if (++s == STAGES) { s = 0; full_parity ^= 1u; }
                 }
+            }
+        }
+    } else if (XF > 0 && warp >= 2 + EPI) {
+        // ------------------------------------------------- operand transform: W hi / lo of theta +- eps_fd p
+        // Both buffers of a stage carry the same 128-byte swizzle at the same alignment, so the element at byte
+        // offset o of the theta tile meets its p at offset o of the p tile, and hi / lo go back to the same places:
+        // the transform is elementwise over the raw bytes and never needs the row / column of an element.
+        constexpr int NT = XF > 0 ? 32 * XF : 32;
+        constexpr int CHUNKS = W_BYTES / 16;      // 16-byte groups per buffer
+        constexpr int PER = CHUNKS / NT;
+        constexpr int BATCH = PER < 4 ? PER : 4;
+        static_assert(CHUNKS % NT == 0 && PER % BATCH == 0, "the transform threads share a buffer evenly");
+        const int t = (int)threadIdx.x - 32 * (2 + EPI);
+        const float eps = *args.eps_fd;
+        // eps == 0 marks the degenerate norm: the weights are theta itself even where p is not finite, so p's
+        // factor is forced to zero by reading p as zero (0 * NaN would not do)
+        const bool degenerate = eps == 0.f;
+        // hi = tf32(w) with round-to-nearest on the integer pipe (two operations; a conversion instruction
+        // issues at a fraction of that rate).  The add can carry a NaN's mantissa into the sign bit and so turn
+        // it into a zero; the fused multiply-add by zero puts it back (0 * w is NaN exactly when w is not finite,
+        // and then so must the operand be).  lo = tf32(w - hi) needs no such care: it multiplies the same
+        // operands as a hi that is already NaN.
+        auto split = [](float w, float& hi, float& lo) {
+            const float h = __uint_as_float((__float_as_uint(w) + 0x1000u) & 0xFFFFE000u);
+            hi = fmaf(0.f, w, h);
+            lo = __uint_as_float((__float_as_uint(w - hi) + 0x1000u) & 0xFFFFE000u);
+        };
+        int s = 0;
+        uint32_t parity = 0;
+        bool ok = true;
+        for (int step = 0; ok; ++step) {
+            int item, kb0, nkb, tpart;
+            if (!next_work(step, item, kb0, nkb, tpart)) break;
+            const float e = (item / tiles_per_branch) ? -eps : eps;
+            for (int kb = 0; kb < nkb; ++kb) {
+                ok = mbar_wait(wfull_bar(s), parity, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) { if (lane == 0) raise_timeout(); break; }
+                float4* th = reinterpret_cast<float4*>(smem_raw + (base + s * STAGE + 2 * A_BYTES - smem_u32(smem_raw))) + t;
+                float4* pp = th + CHUNKS;
+                // software pipeline: the next batch's loads are issued before this batch's stores (the two never
+                // touch the same 16 bytes, which the compiler cannot know)
+                float4 vt[BATCH], vp[BATCH];
+#pragma unroll
+                for (int j = 0; j < BATCH; ++j) {
+                    vt[j] = th[j * NT];
+                    vp[j] = pp[j * NT];
+                }
+#pragma unroll 1
+                for (int j0 = 0; j0 < PER; j0 += BATCH) {
+                    float4 h[BATCH], l[BATCH];
+#pragma unroll
+                    for (int j = 0; j < BATCH; ++j) {
+                        const float4 q = degenerate ? make_float4(0.f, 0.f, 0.f, 0.f) : vp[j];
+                        split(fmaf(e, q.x, vt[j].x), h[j].x, l[j].x);
+                        split(fmaf(e, q.y, vt[j].y), h[j].y, l[j].y);
+                        split(fmaf(e, q.z, vt[j].z), h[j].z, l[j].z);
+                        split(fmaf(e, q.w, vt[j].w), h[j].w, l[j].w);
+                    }
+                    if (j0 + BATCH < PER) {
+#pragma unroll
+                        for (int j = 0; j < BATCH; ++j) {
+                            vt[j] = th[(j0 + BATCH + j) * NT];
+                            vp[j] = pp[(j0 + BATCH + j) * NT];
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < BATCH; ++j) {
+                        th[(j0 + j) * NT] = h[j];
+                        pp[(j0 + j) * NT] = l[j];
+                    }
+                }
+                // these writes, made through the generic proxy, must be visible to the tensor core's reads
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) {
+                    if (PAIR) mbar_arrive_cluster(ready_bar(s) & kPeerBitMask); else mbar_arrive(ready_bar(s));
+                }
+                if (++s == STAGES) { s = 0; parity ^= 1u; }
             }
         }
     } else {
@@ -1002,21 +1130,21 @@ const CUtensorMap* cached_map(TcState* st, const float* base, int ld, int64_t ro
     return &st->maps[slot];
 }
 
-template <int BN, bool PAIR, int EPI>
+template <int BN, bool PAIR, int EPI, int XF>
 cudaError_t tc_prepare_kernel() {
-    return cudaFuncSetAttribute(gemm_tf32x3_kernel<BN, PAIR, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(gemm_tf32x3_kernel<BN, PAIR, EPI, XF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 smem_bytes(PAIR ? BN / 2 : BN));
 }
 
 // Launches the persistent kernel on min(work items, co-resident CTAs or CTA pairs) units.
-template <int BN, bool PAIR, int EPI>
+template <int BN, bool PAIR, int EPI, int XF>
 cudaError_t launch_tc(const CUtensorMap* const maps[4], const TcArgs& a, int items, int max_units, bool tail_ok,
                       cudaStream_t st, size_t ws_floats = 0, int tail_flags = 0) {
     const int ks = PAIR ? 1 : a.ksplit;
     constexpr int kSmem = smem_bytes(PAIR ? BN / 2 : BN);
     if (max_units < 1) return cudaErrorLaunchOutOfResources;
     if (ks > 1)  // one tile per cluster of ks CTAs
-        return launch_clustered(ks, gemm_tf32x3_kernel<BN, PAIR, EPI>, dim3(items * ks), dim3(threads_for(EPI)),
+        return launch_clustered(ks, gemm_tf32x3_kernel<BN, PAIR, EPI, XF>, dim3(items * ks), dim3(threads_for(EPI, XF)),
                                 (size_t)kSmem, st, *maps[0], *maps[1], *maps[2], *maps[3], a);
     const int units = items < max_units ? items : max_units;
     TcArgs b = a;
@@ -1032,8 +1160,8 @@ cudaError_t launch_tc(const CUtensorMap* const maps[4], const TcArgs& a, int ite
             b.tail_tiles = tail;
         }
     }
-    return launch_clustered(PAIR ? 2 : 1, gemm_tf32x3_kernel<BN, PAIR, EPI>, dim3(units * (PAIR ? 2 : 1)),
-                            dim3(threads_for(EPI)), (size_t)kSmem, st, *maps[0], *maps[1], *maps[2], *maps[3], b);
+    return launch_clustered(PAIR ? 2 : 1, gemm_tf32x3_kernel<BN, PAIR, EPI, XF>, dim3(units * (PAIR ? 2 : 1)),
+                            dim3(threads_for(EPI, XF)), (size_t)kSmem, st, *maps[0], *maps[1], *maps[2], *maps[3], b);
 }
 
 inline int round_up32(int x) { return (x + 31) & ~31; }
@@ -1090,13 +1218,16 @@ cudaError_t tc_state_create(sama_ctx* ctx) {
     if (const char* e = std::getenv("SAMA_TC_TAIL")) st->no_tail = e[0] == '0';
     if (const char* e = std::getenv("SAMA_TC_GROUP")) st->group = std::atoi(e);
     cudaError_t e;
-    if ((e = tc_prepare_kernel<256, true, 8>()) != cudaSuccess) return e;
-    if ((e = tc_prepare_kernel<128, false, 8>()) != cudaSuccess) return e;
-    if ((e = tc_prepare_kernel<64, false, 8>()) != cudaSuccess) return e;
-    if ((e = tc_prepare_kernel<16, false, 4>()) != cudaSuccess) return e;
+    if ((e = tc_prepare_kernel<256, true, 8, 0>()) != cudaSuccess) return e;
+    if ((e = tc_prepare_kernel<128, false, 8, 0>()) != cudaSuccess) return e;
+    if ((e = tc_prepare_kernel<64, false, 8, 0>()) != cudaSuccess) return e;
+    if ((e = tc_prepare_kernel<16, false, 4, 0>()) != cudaSuccess) return e;
+    if ((e = tc_prepare_kernel<256, true, 8, kXf>()) != cudaSuccess) return e;
+    if ((e = tc_prepare_kernel<128, false, 8, kXf>()) != cudaSuccess) return e;
+    if ((e = tc_prepare_kernel<64, false, 8, kXf>()) != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * (ctx->sm_count / 2));
-    cfg.blockDim = dim3(threads_for(8));
+    cfg.blockDim = dim3(threads_for(8, kXf));
     cfg.dynamicSmemBytes = smem_bytes(128);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1106,7 +1237,7 @@ cudaError_t tc_state_create(sama_ctx* ctx) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int clusters = 0;
-    if ((e = cudaOccupancyMaxActiveClusters(&clusters, gemm_tf32x3_kernel<256, true, 8>, &cfg)) != cudaSuccess) return e;
+    if ((e = cudaOccupancyMaxActiveClusters(&clusters, gemm_tf32x3_kernel<256, true, 8, kXf>, &cfg)) != cudaSuccess) return e;
     st->pair_units = clusters < ctx->sm_count / 2 ? clusters : ctx->sm_count / 2;
     return cudaSuccess;
 }
@@ -1177,10 +1308,16 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     const int wrows = pair ? bn / 2 : bn;
     const int a_box = L.M < BM ? L.M : BM, w_box = L.N < wrows ? L.N : wrows;
     const int64_t a_slab = (int64_t)L.M * Kp;
+    // W operands: the pre-split copy, or (w_theta given) this layer's block of theta and of p themselves, rows
+    // of K floats, from which the kernel forms them; columns beyond K read as zero
+    const bool xf = L.w_theta != nullptr;
+    if (xf && (narrow_last || !L.w_p || !L.eps_fd || L.K < BKF || (L.K & 3) || nbr != 2)) return cudaErrorInvalidValue;
     const CUtensorMap* maps[4] = {cached_map(ts, L.a_hi, Kp, L.M, a_slabs, a_box, a_slab),
                                   cached_map(ts, L.a_lo, Kp, L.M, a_slabs, a_box, a_slab),
-                                  cached_map(ts, L.w_hi, Kp, L.N, nbr, w_box, L.w_slab),
-                                  cached_map(ts, L.w_lo, Kp, L.N, nbr, w_box, L.w_slab)};
+                                  xf ? cached_map(ts, L.w_theta, L.K, L.N, 1, w_box, (int64_t)L.N * L.K)
+                                     : cached_map(ts, L.w_hi, Kp, L.N, nbr, w_box, L.w_slab),
+                                  xf ? cached_map(ts, L.w_p, L.K, L.N, 1, w_box, (int64_t)L.N * L.K)
+                                     : cached_map(ts, L.w_lo, Kp, L.N, nbr, w_box, L.w_slab)};
     if (!maps[0] || !maps[1] || !maps[2] || !maps[3]) return cudaErrorInvalidValue;
     TcArgs a;
     a.bias[0] = L.bias[0];
@@ -1200,7 +1337,10 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     a.both = L.both;
     a.mask = L.mask;
     a.ldm = L.ldm;
-    a.tx_bytes = (uint32_t)(2 * a_box * BKF * 4 + 2 * w_box * BKF * 4) * (pair ? 2u : 1u);  // a pair's barrier counts both CTAs' copies
+    // a pair's barrier counts both CTAs' copies
+    a.tx_bytes = (uint32_t)(2 * a_box * BKF * 4 + (xf ? 0 : 2 * w_box * BKF * 4)) * (pair ? 2u : 1u);
+    a.w_tx_bytes = (uint32_t)(2 * w_box * BKF * 4);
+    a.eps_fd = L.eps_fd;
     a.status = &ctx->scalars->status;
     a.tiles_m = pair ? (L.M + 2 * BM - 1) / (2 * BM) : (L.M + BM - 1) / BM;
     a.tiles_n = (L.N + bn - 1) / bn;
@@ -1222,12 +1362,19 @@ cudaError_t launch_gemm_tf32x3(sama_ctx* ctx, const TcLayer& L, cudaStream_t st)
     // its small kernels (the direct gradient, see run_meta_grad_tc).
     PdlScope pdl(pdl_enabled() ? 1 : 0);
     // eight epilogue warps (two per lane quarter, each taking half of the columns) except on the 16-wide tile
+    if (xf) {
+        if (pair)
+            return launch_tc<256, true, 8, kXf>(maps, a, items, ts->pair_units, !ts->no_tail, st, ctx->tc_ws_floats,
+                                                ctx->tc_flags ? kTcFlags : 0);
+        if (bn == 64) return launch_tc<64, false, 8, kXf>(maps, a, items, sms, false, st);
+        return launch_tc<128, false, 8, kXf>(maps, a, items, sms, false, st);
+    }
     if (pair)
-        return launch_tc<256, true, 8>(maps, a, items, ts->pair_units, !ts->no_tail, st, ctx->tc_ws_floats,
-                                       ctx->tc_flags ? kTcFlags : 0);
-    if (bn == 16) return launch_tc<16, false, 4>(maps, a, items, sms, false, st);
-    if (bn == 64) return launch_tc<64, false, 8>(maps, a, items, sms, false, st);
-    return launch_tc<128, false, 8>(maps, a, items, sms, false, st);
+        return launch_tc<256, true, 8, 0>(maps, a, items, ts->pair_units, !ts->no_tail, st, ctx->tc_ws_floats,
+                                          ctx->tc_flags ? kTcFlags : 0);
+    if (bn == 16) return launch_tc<16, false, 4, 0>(maps, a, items, sms, false, st);
+    if (bn == 64) return launch_tc<64, false, 8, 0>(maps, a, items, sms, false, st);
+    return launch_tc<128, false, 8, 0>(maps, a, items, sms, false, st);
 }
 
 }  // namespace sama

@@ -208,11 +208,29 @@ bool fused_head_only_model(const sama_mlp_t* mlp) {
     return mlp->n_layers == 1 && head_applicable(mlp->dims[1]);
 }
 
+// Layers of the tensor-core forward whose W operands the product kernel can form itself from theta and p
+// (bit l set), given that the preconditions of the fused perturbation sweep hold (16-byte aligned theta and p,
+// every weight block at a multiple of 4 with K % 4 == 0): every matrix-product layer with K >= 32 except a
+// narrow last one, which takes the 16-wide tile.
+uint32_t wfuse_mask(const sama_ctx* ctx, const sama_mlp_t* mlp) {
+    if (ctx->gemm_mode != 3) return 0u;
+    const bool fused_head = head_applicable(mlp->dims[mlp->n_layers]);
+    const int L = fused_head ? mlp->n_layers - 1 : mlp->n_layers;
+    uint32_t mask = 0u;
+    for (int l = 0; l < L; ++l) {
+        const bool narrow_last = (l + 1 == L) && mlp->dims[l + 1] <= 16;
+        if (!narrow_last && mlp->dims[l] >= 32) mask |= 1u << l;
+    }
+    return mask;
+}
+
 // Forward pass of both branches on the tensor cores (3xTF32).  Operands are TF32 hi/lo pairs: X is split
 // here, hidden activations by the epilogue that produces them, and the weights either by the fused
-// perturbation sweep (w_presplit) or here, layer by layer.
+// perturbation sweep (w_presplit), or by the product kernel itself from theta and p (layers in `wfuse`, which
+// implies w_presplit for the rest), or here, layer by layer.
 int run_forward_tc(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const float* theta_minus,
-                   const float* X, int32_t B, bool w_presplit, bool x_presplit, bool fused_head, cudaStream_t st) {
+                   const float* X, int32_t B, bool w_presplit, bool x_presplit, bool fused_head, cudaStream_t st,
+                   const float* theta0 = nullptr, const float* p = nullptr, uint32_t wfuse = 0u) {
     // with a fused head the last layer is not a matrix product here, and the layer before it
     // leaves fp32 activations (ReLU applied) in the context's activation buffer
     const int L = fused_head ? mlp->n_layers - 1 : mlp->n_layers;
@@ -241,6 +259,11 @@ int run_forward_tc(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus
         t.w_hi = w_hi + lay.s_off[l];
         t.w_lo = w_lo + lay.s_off[l];
         t.w_slab = lay.slab;
+        if ((wfuse >> l) & 1u) {
+            t.w_theta = theta0 + lay.w_off[l];
+            t.w_p = p + lay.w_off[l];
+            t.eps_fd = &ctx->scalars->eps_fd;
+        }
         // biases: from the compact slab the fused perturbation sweep filled, else straight from theta+-
         t.bias[0] = w_presplit ? ctx->pm_small + lay.b_off[l] : theta_plus + lay.w_off[l] + lay.w_cnt[l];
         t.bias[1] = w_presplit ? ctx->pm_small + lay.small + lay.b_off[l] : theta_minus + lay.w_off[l] + lay.w_cnt[l];
@@ -265,13 +288,14 @@ int run_forward_tc(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus
 int run_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const float* theta_minus,
            const float* X, const int32_t* y, const float* lambda, int32_t B, const float* eps_fd,
            float* metagrad_out, float* loss_plus_out, float* loss_minus_out, cudaStream_t st,
-           bool w_presplit = false, bool x_presplit = false) {
+           bool w_presplit = false, bool x_presplit = false, const float* theta0 = nullptr, const float* p = nullptr,
+           uint32_t wfuse = 0u) {
     const int L = mlp->n_layers;
     const int C = mlp->dims[L];
     const bool fits = tc_fits(ctx, mlp, B);
-    if (ctx->gemm_mode == 2 && !fits) return SAMA_ERR_SIZE;
+    if (ctx->gemm_mode >= 2 && !fits) return SAMA_ERR_SIZE;
     const bool use_tc = ctx->gemm_mode != 1 && fits;
-    ctx->last_forward_path = use_tc ? 2 : 1;
+    ctx->last_forward_path = use_tc ? (wfuse ? 3 : 2) : 1;
     const bool fused_head = head_applicable(C);
     const float* eps = eps_fd ? eps_fd : &ctx->scalars->eps_fd;
     float* diff_out = ctx->rw_buf ? ctx->rw_buf + 4 * (size_t)ctx->max_batch : nullptr;
@@ -280,7 +304,8 @@ int run_fd(sama_ctx* ctx, const sama_mlp_t* mlp, const float* theta_plus, const 
     int ld_in = mlp->dims[0];
 
     if (use_tc) {
-        const int rc = run_forward_tc(ctx, mlp, theta_plus, theta_minus, X, B, w_presplit, x_presplit, fused_head, st);
+        const int rc = run_forward_tc(ctx, mlp, theta_plus, theta_minus, X, B, w_presplit, x_presplit, fused_head, st,
+                                      theta0, p, wfuse);
         if (rc != SAMA_OK) return rc;
         if (n_gemm > 0) {
             float* out = fused_head ? ctx->act[0] : ctx->logits;
@@ -563,9 +588,12 @@ int sama_step(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* thet
     if (!guard.ok) return SAMA_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;
     // With the tensor-core forward, the perturbation sweep also emits the TF32 operand split of W+-.
-    const SplitLayout lay = make_split_layout(mlp);
+    SplitLayout lay = make_split_layout(mlp);
     const bool fused = ctx->gemm_mode != 1 && tc_fits(ctx, mlp, B) &&
                        perturb_split_applicable(lay, theta, p_out, theta_plus, theta_minus);
+    // ... except for the layers whose product kernel forms them itself from theta and p
+    const uint32_t wfuse = fused ? wfuse_mask(ctx, mlp) : 0u;
+    lay.skip_w = wfuse;
     // ... and for a model small enough, adaptation and norm join it in one launch
     const bool one_launch = fused && aligned(g_meta, 16) && (c.identity || (aligned(m, 16) && aligned(s, 16))) &&
                             (c.identity || !g_base || aligned(g_base, 16)) && fused_sweep_applicable(ctx, n);
@@ -623,7 +651,7 @@ int sama_step(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* thet
                                       nullptr, st));
     }
     return run_fd(ctx, mlp, theta_plus, theta_minus, X, y, lambda, B, nullptr, metagrad_out, loss_plus_out,
-                  loss_minus_out, st, fused, x_fused);
+                  loss_minus_out, st, fused, x_fused, theta, p_out, wfuse);
 }
 
 int sama_fd_metagrad_reweight(sama_ctx* ctx, int32_t B, const float* loss_plus, const float* loss_minus,
@@ -854,7 +882,7 @@ int sama_last_cuda_error(sama_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0;
 
 int sama_set_gemm_mode(sama_ctx* ctx, int mode) {
     if (!ctx) return SAMA_ERR_NULL;
-    if (mode < 0 || mode > 2) return SAMA_ERR_PARAM;
+    if (mode < 0 || mode > 3) return SAMA_ERR_PARAM;
     ctx->gemm_mode = mode;
     return SAMA_OK;
 }

@@ -53,6 +53,8 @@ struct SplitLayout {
     int head_layer;             // index of the layer whose fp32 weights are kept (the fused head's), or -1
     int64_t head_cnt;           // its weight count (at offset 0 of the small slab), else 0
     int64_t small;              // floats per small slab
+    // Bit l set: the forward forms layer l's W operands itself from theta and p, so the sweep writes none for it.
+    uint32_t skip_w;
 };
 
 // The batch X as an extra job of the fused perturbation sweep: its TF32 hi/lo split, rows padded to ld_out.
@@ -84,7 +86,7 @@ struct sama_ctx {
     int32_t max_batch;
     int32_t max_width;    // widest hidden layer the forward workspace covers, 0 if none
     int32_t max_classes;  // largest d_L covered, 0 if the context has no forward workspace
-    int gemm_mode;        // 0 auto, 1 ffma, 2 3xTF32
+    int gemm_mode;        // 0 auto, 1 ffma, 2 3xTF32, 3 3xTF32 with W+- formed in the product kernel's operand stage
     int last_cuda_error;
     int fused_sweep_blocks;  // co-resident blocks per SM of the fused sweep kernel on this device (0: not yet asked, -1: unavailable)
     int no_fused_sweep;      // SAMA_NO_FUSED_SWEEP=1 (experiment switch, read at sama_create)
@@ -261,6 +263,11 @@ struct TcLayer {
     int both = 0;                // hidden layer that also stores fp32 to out_f32
     const float* mask = nullptr; // [M][ldm]: zero the result where mask <= 0
     int ldm = 0;
+    // When w_theta is given, w_hi / w_lo are ignored: the kernel forms the operands of theta +- eps_fd p itself
+    // from this layer's weights inside theta and p ([N][K] fp32; 16-byte aligned, K % 4 == 0, K >= 32).
+    const float* w_theta = nullptr;
+    const float* w_p = nullptr;
+    const float* eps_fd = nullptr;  // device
 };
 // hi/lo of the TRANSPOSE of a dense fp32 matrix [rows][cols]: out [cols][round32(rows)], zero padded
 cudaError_t launch_split_transpose_tf32(sama_ctx* ctx, const float* src, int64_t rows, int cols, float* hi, float* lo,

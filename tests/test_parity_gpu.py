@@ -170,6 +170,9 @@ RAGGED = [((12, 5), 1), ((33, 17, 12, 6), 7), ((100, 50, 3), 129), ((257, 130, 6
 
 # 1 = fp32 FMA on the CUDA cores, 2 = tensor cores (three TF32 products per fp32 product)
 GEMM_MODES = [1, 2]
+# sama_step also has mode 3: tensor cores, with the weights of both branches formed in the product kernel's
+# operand stage from theta and p instead of being read as a pre-split copy
+STEP_MODES = [1, 2, 3]
 
 
 @pytest.mark.parametrize("gemm_mode", GEMM_MODES)
@@ -286,14 +289,14 @@ def check_step(cfg, w, adam, alpha, rows=None, use_gbase=True, gemm_mode=0, key=
     return e
 
 
-@pytest.mark.parametrize("gemm_mode", GEMM_MODES)
+@pytest.mark.parametrize("gemm_mode", STEP_MODES)
 @pytest.mark.parametrize("alpha", [1e-2, 1.0])
 def test_step_parity_tiny(alpha, gemm_mode):
     cfg = W.CONFIGS["tiny"]
     check_step(cfg, W.mlp_workload(cfg, 0), B.Adam(), alpha, gemm_mode=gemm_mode, key=("tiny", alpha))
 
 
-@pytest.mark.parametrize("gemm_mode", GEMM_MODES)
+@pytest.mark.parametrize("gemm_mode", STEP_MODES)
 def test_step_parity_tiny_variants(gemm_mode):
     cfg = W.CONFIGS["tiny"]
     w = W.mlp_workload(cfg, 0)
@@ -308,14 +311,14 @@ def test_step_parity_tiny_variants(gemm_mode):
     check_step(cfg, w, B.Adam(bias_correction=False), 1.0, use_gbase=False, gemm_mode=gemm_mode, key=("tiny", "nobias"))
 
 
-@pytest.mark.parametrize("gemm_mode", GEMM_MODES)
+@pytest.mark.parametrize("gemm_mode", STEP_MODES)
 @pytest.mark.parametrize("dims,batch", RAGGED[1:])
 def test_step_parity_ragged(dims, batch, gemm_mode):
     cfg, w = W.custom_mlp(dims, batch, seed=3 + sum(dims))
     check_step(cfg, w, B.Adam(), 1e-2, gemm_mode=gemm_mode, key=("ragged", dims, batch))
 
 
-@pytest.mark.parametrize("gemm_mode", GEMM_MODES)
+@pytest.mark.parametrize("gemm_mode", STEP_MODES)
 def test_step_parity_mlp3072(gemm_mode):
     cfg = W.CONFIGS["mlp3072"]
     w = W.mlp_workload(cfg, 0)
@@ -323,7 +326,7 @@ def test_step_parity_mlp3072(gemm_mode):
     check_step(cfg, w, B.Adam(), 1.0, rows=np.arange(0, cfg.batch, 8), gemm_mode=gemm_mode, key=("mlp3072", 1.0))
 
 
-@pytest.mark.parametrize("gemm_mode", GEMM_MODES)
+@pytest.mark.parametrize("gemm_mode", STEP_MODES)
 def test_step_parity_head1024(gemm_mode):
     cfg = W.CONFIGS["head1024"]
     w = W.mlp_workload(cfg, 0)
@@ -331,7 +334,7 @@ def test_step_parity_head1024(gemm_mode):
     check_step(cfg, w, B.Adam(), 1.0, rows=np.arange(0, cfg.batch, 64), gemm_mode=gemm_mode, key=("head1024", 1.0))
 
 
-@pytest.mark.parametrize("gemm_mode", GEMM_MODES)
+@pytest.mark.parametrize("gemm_mode", STEP_MODES)
 def test_step_parity_wide4096_sampled(gemm_mode):
     """Full-size launch; the checker evaluates a sample of the rows (each output
     depends only on its own row given theta+-, which are compared in full)."""
@@ -342,7 +345,7 @@ def test_step_parity_wide4096_sampled(gemm_mode):
     check_step(cfg, w, B.Adam(), 1.0, rows=rows[::2], gemm_mode=gemm_mode, key=("wide4096", 1.0))
 
 
-@pytest.mark.parametrize("gemm_mode", GEMM_MODES)
+@pytest.mark.parametrize("gemm_mode", STEP_MODES)
 def test_step_is_bitwise_reproducible(gemm_mode):
     """Fixed reduction orders everywhere (norm partials, split-K partial tiles): repeated steps agree bit for bit."""
     for cfg, w in [(W.CONFIGS["tiny"], W.mlp_workload(W.CONFIGS["tiny"], 0)), W.custom_mlp((40, 200, 72, 24), 257, seed=5),
@@ -385,7 +388,7 @@ def test_shared_tail_tiles_of_the_pair_kernel():
     assert np.array_equal(a["metagrad"], b["metagrad"]) and np.array_equal(a["loss_plus"], c["loss_plus"])
 
 
-@pytest.mark.parametrize("gemm_mode", GEMM_MODES)
+@pytest.mark.parametrize("gemm_mode", STEP_MODES)
 @pytest.mark.parametrize("dims,batch", [((784, 256, 10), 128), ((40, 200, 72, 24), 257), ((64, 64, 64, 16), 300),
                                         ((33, 17, 12, 6), 7)])
 def test_step_without_theta_outputs(dims, batch, gemm_mode):
@@ -402,6 +405,33 @@ def test_step_without_theta_outputs(dims, batch, gemm_mode):
             assert got["eps_fd"] == full["eps_fd"] and got["status"] == 0
             for k, want in (("theta_plus", want_plus), ("theta_minus", want_minus)):
                 assert np.array_equal(got[k], full[k]) if want else np.all(np.isnan(got[k]))
+
+
+@pytest.mark.parametrize("dims,batch", [((784, 256, 10), 128), ((40, 200, 72, 24), 257), ((3072, 1024, 1024, 10), 512),
+                                        ((300, 2304, 40), 1200), ((512, 2560, 40), 1280)])
+def test_weights_formed_in_the_operand_stage_match_the_presplit_copy(dims, batch):
+    """Mode 3 forms hi / lo of theta +- eps_fd p inside the product kernel (theta and p tiles land in shared
+    memory and are replaced in place); mode 2 reads the same numbers from the copy the perturbation sweep wrote.
+    Same operands, same order of products: every output agrees bit for bit, on single-CTA tiles, clusters that
+    split the contraction, CTA pairs with shared tail tiles, and contractions that end inside a k-block (columns
+    beyond K read as zero).  A non-finite weight still shows."""
+    cfg, w = W.custom_mlp(dims, batch, seed=21 + batch)
+    out = {}
+    for mode in (2, 3):
+        with Ctx(cfg.n_params, cfg.batch, cfg.dims, mode) as ctx:
+            out[mode] = run_step(ctx, cfg, w, B.Adam(), 1e-2)
+            assert B.sama_last_forward_path(ctx.h) == mode and out[mode]["status"] == 0
+            if mode == 3:
+                again = run_step(ctx, cfg, w, B.Adam(), 1e-2, want_plus=False, want_minus=False)
+                bad = dict(w)
+                bad["theta"] = w["theta"].copy()
+                bad["theta"][5] = np.nan
+                poisoned = run_step(ctx, cfg, bad, B.Adam(), 1e-2)
+    for k in ("p", "theta_plus", "theta_minus", "metagrad", "loss_plus", "loss_minus"):
+        assert np.array_equal(out[2][k], out[3][k]), k
+    for k in ("metagrad", "loss_plus", "loss_minus"):
+        assert np.array_equal(again[k], out[3][k]), k
+    assert np.isnan(poisoned["loss_plus"]).all() and np.isnan(poisoned["loss_minus"]).all()
 
 
 @pytest.mark.parametrize("name", ["tiny", "mlp3072"])
