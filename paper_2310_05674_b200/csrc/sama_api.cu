@@ -592,7 +592,9 @@ int sama_step(sama_ctx* ctx, const sama_mlp_t* mlp, int64_t n, const float* thet
     const bool fused = ctx->gemm_mode != 1 && tc_fits(ctx, mlp, B) &&
                        perturb_split_applicable(lay, theta, p_out, theta_plus, theta_minus);
     // ... except for the layers whose product kernel forms them itself from theta and p
-    const uint32_t wfuse = fused ? wfuse_mask(ctx, mlp) : 0u;
+    // (not when theta+ or theta- is written over theta, the in-place nudge: the products read theta after the sweep)
+    const bool theta_kept = !overlaps(theta_plus, nb, theta, nb) && !overlaps(theta_minus, nb, theta, nb);
+    const uint32_t wfuse = (fused && theta_kept) ? wfuse_mask(ctx, mlp) : 0u;
     lay.skip_w = wfuse;
     // ... and for a model small enough, adaptation and norm join it in one launch
     const bool one_launch = fused && aligned(g_meta, 16) && (c.identity || (aligned(m, 16) && aligned(s, 16))) &&

@@ -427,8 +427,20 @@ def test_weights_formed_in_the_operand_stage_match_the_presplit_copy(dims, batch
                 bad["theta"] = w["theta"].copy()
                 bad["theta"][5] = np.nan
                 poisoned = run_step(ctx, cfg, bad, B.Adam(), 1e-2)
+                # the in-place nudge (theta- written over theta, Sec. 3.2): theta is gone by the time the products
+                # run, so this call reads the pre-split copy after all
+                t = {k: dev(w[k]) for k in ["theta", "m", "s", "g_base", "g_meta", "X", "y", "lam"]}
+                fl = lambda k: torch.empty(k, dtype=torch.float32, device=DEV)
+                p_o, mg_o = fl(cfg.n_params), fl(cfg.batch)
+                B.sama_step(ctx.h, ctx.mlp, cfg.n_params, t["theta"], t["m"], t["s"], t["g_base"], t["g_meta"], B.Adam(),
+                            1e-2, t["X"], t["y"], t["lam"], cfg.batch, p_o, None, t["theta"], mg_o, None, None)
+                torch.cuda.synchronize()
+                assert B.sama_last_forward_path(ctx.h) == 2
+                nudged = {"theta_minus": t["theta"].cpu().numpy(), "metagrad": mg_o.cpu().numpy()}
     for k in ("p", "theta_plus", "theta_minus", "metagrad", "loss_plus", "loss_minus"):
         assert np.array_equal(out[2][k], out[3][k]), k
+    for k in ("theta_minus", "metagrad"):
+        assert np.array_equal(nudged[k], out[3][k]), k
     for k in ("metagrad", "loss_plus", "loss_minus"):
         assert np.array_equal(again[k], out[3][k]), k
     assert np.isnan(poisoned["loss_plus"]).all() and np.isnan(poisoned["loss_minus"]).all()
