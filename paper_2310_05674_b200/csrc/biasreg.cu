@@ -7,10 +7,16 @@
 //   central difference (Eq. 5) of g_lambda(w) = dL_base/dlambda = -2 beta (w - lambda):
 //                             metagrad = -[g_lambda(w+) - g_lambda(w-)] / (2 eps_fd)
 //
-// The direct gradient reads X' once from HBM: a block takes a contiguous run of rows, eight at a time; each warp
-// forms one residual r_i = x_i . w - y_i, then all threads add r_i x_i into the block's partial gradient in
-// shared memory (the rows come back from L1 / L2).  A second small kernel adds the blocks' partials column by
-// column in block order.  Accumulation is double throughout; nothing depends on scheduling.
+// The direct gradient is two sweeps over X', each at streaming rate, instead of one that keeps a block's partial
+// gradient in shared memory (that form needs two block-wide phases per handful of rows and is latency-bound):
+//   1. residuals: one warp per row forms r_i = x_i . w - y_i (every load of a row segment in flight at once; the
+//      sum kept as pairs of floats that carry a double's precision) and stores it in double;
+//   2. column sums: a block takes a strip of 1024 columns (one float4 per thread) and a chunk of rows, reads the
+//      strip of each row (4 KB, contiguous; the chunks run from the last rows backwards, so that what the first
+//      sweep left in L2 is read from there), and adds
+//      r_i x_i into four double accumulators per thread; the chunk's partial goes to global memory.
+// A third small kernel adds the chunks' partials column by column in chunk order.  Accumulation carries a
+// double's precision throughout; nothing depends on scheduling.
 #include "sama_internal.h"
 
 namespace sama {
@@ -18,122 +24,170 @@ namespace sama {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kRows = kThreads / 32;  // rows in flight per block = warps
+constexpr int kWarps = kThreads / 32;
 
-// VEC: d % 4 == 0 and 16-byte aligned X', w: 16-byte loads, four times as many bytes in flight per thread.
+// VEC: d % 4 == 0 and 16-byte aligned X', w: 16-byte loads, kSeg of them per lane in flight before the first is
+// used (a row is a chain of dependent steps for its warp, so the loads in flight per lane set the pace).
+constexpr int kSeg = 8;
+
+// One more term x w of a dot product kept as an unevaluated sum s + e of two floats: the product is exact as
+// ph + pl (fused multiply-add), s + ph is exact as t + (rounding error) by Knuth's two-sum, and the small parts
+// gather in e.  The result carries about 2^-45 of the sum of |x w|, like a double accumulator, without the
+// float-to-double conversions (two per term), which this device issues slowly: measured 37 -> 29 us for the
+// sweep below at d = 4096, n' = 8192, with results equal to the double form's to 12 digits.
+// (Intrinsics, so that no multiply is contracted into a neighbouring add.)
+__device__ __forceinline__ void dot_step(float& s, float& e, float x, float w) {
+    const float ph = __fmul_rn(x, w);
+    const float pl = __fmaf_rn(x, w, -ph);
+    const float t = __fadd_rn(s, ph);
+    const float z = __fsub_rn(t, s);
+    const float err = __fadd_rn(__fsub_rn(s, __fsub_rn(t, z)), __fsub_rn(ph, z));
+    e = __fadd_rn(e, __fadd_rn(err, pl));
+    s = t;
+}
+__device__ __forceinline__ void dot_step4(float& s, float& e, float4 x, float4 w) {
+    dot_step(s, e, x.x, w.x);
+    dot_step(s, e, x.y, w.y);
+    dot_step(s, e, x.z, w.z);
+    dot_step(s, e, x.w, w.w);
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(kThreads, 4)
+biasreg_residual_kernel(int d, int n_val, const float* __restrict__ Xv, const float* __restrict__ yv,
+                        const float* __restrict__ w, double* __restrict__ res) {
+    const int lane = threadIdx.x & 31;
+    const int warp = blockIdx.x * kWarps + (threadIdx.x >> 5), n_warps = gridDim.x * kWarps;
+    for (int i = warp; i < n_val; i += n_warps) {
+        const float* x = Xv + (int64_t)i * d;
+        double r;
+        if (VEC) {
+            const float4* x4 = reinterpret_cast<const float4*>(x);
+            const float4* w4 = reinterpret_cast<const float4*>(w);
+            const int q = d >> 2;
+            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f, e0 = 0.f, e1 = 0.f, e2 = 0.f, e3 = 0.f;   // four independent chains
+            for (int c0 = 0; c0 < q; c0 += 32 * kSeg) {
+                float4 a[kSeg];
+#pragma unroll
+                for (int k = 0; k < kSeg; ++k) {
+                    const int c = c0 + lane + 32 * k;
+                    a[k] = c < q ? __ldg(x4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int k = 0; k < kSeg; k += 4) {
+                    float4 b[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int c = c0 + lane + 32 * (k + j);
+                        b[j] = c < q ? __ldg(w4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);   // w: 4 d bytes, from L1
+                    }
+                    dot_step4(s0, e0, a[k], b[0]);
+                    dot_step4(s1, e1, a[k + 1], b[1]);
+                    dot_step4(s2, e2, a[k + 2], b[2]);
+                    dot_step4(s3, e3, a[k + 3], b[3]);
+                }
+            }
+            r = (((double)s0 + (double)e0) + ((double)s1 + (double)e1)) + (((double)s2 + (double)e2) + ((double)s3 + (double)e3));
+        } else {
+            double r0 = 0.0, r1 = 0.0, r2 = 0.0, r3 = 0.0;
+            int c = lane;
+            for (; c + 96 < d; c += 128) {
+                r0 = fma((double)x[c], (double)w[c], r0);
+                r1 = fma((double)x[c + 32], (double)w[c + 32], r1);
+                r2 = fma((double)x[c + 64], (double)w[c + 64], r2);
+                r3 = fma((double)x[c + 96], (double)w[c + 96], r3);
+            }
+            for (; c < d; c += 32) r0 = fma((double)x[c], (double)w[c], r0);
+            r = (r0 + r1) + (r2 + r3);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) r += __shfl_xor_sync(0xffffffffu, r, o);
+        if (lane == 0) res[i] = r - (double)yv[i];
+    }
+}
+
+// Block (strip, chunk): partial[chunk][c] = sum over the chunk's rows, in row order, of r_i x_ic for the strip's
+// columns; the strip-0 block also leaves the chunk's sum of r_i^2 in column d (the meta loss).
 template <bool VEC>
 __global__ void __launch_bounds__(kThreads)
-biasreg_partials_kernel(int d, int n_val, const float* __restrict__ Xv, const float* __restrict__ yv,
-                        const float* __restrict__ w, double* __restrict__ partials) {
-    extern __shared__ double g_s[];        // [d] partial gradient, then [kRows] residuals
-    double* r_s = g_s + d;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int c = threadIdx.x; c < d; c += kThreads) g_s[c] = 0.0;
-    // this block's rows: a contiguous run, the same for every launch of this shape
-    const int per = (n_val + gridDim.x - 1) / gridDim.x;
-    const int row0 = blockIdx.x * per, row1 = min(n_val, row0 + per);
-    double sq = 0.0;                        // sum of r_i^2 over this warp's rows (lane 0)
-    __syncthreads();
-    for (int base = row0; base < row1; base += kRows) {
-        const int i = base + warp;
-        double r = 0.0;
-        if (i < row1) {
-            const float* x = Xv + (int64_t)i * d;
-            double r0 = 0.0, r1 = 0.0, r2 = 0.0, r3 = 0.0;   // four independent chains
-            if (VEC) {
-                const float4* x4 = reinterpret_cast<const float4*>(x);
-                const float4* w4 = reinterpret_cast<const float4*>(w);
-                const int q = d >> 2;
-                int c = lane;
-                for (; c + 96 < q; c += 128) {
-                    const float4 a0 = __ldg(x4 + c), a1 = __ldg(x4 + c + 32), a2 = __ldg(x4 + c + 64), a3 = __ldg(x4 + c + 96);
-                    const float4 b0 = __ldg(w4 + c), b1 = __ldg(w4 + c + 32), b2 = __ldg(w4 + c + 64), b3 = __ldg(w4 + c + 96);
-                    r0 = fma((double)a0.x, (double)b0.x, r0); r0 = fma((double)a0.y, (double)b0.y, r0);
-                    r0 = fma((double)a0.z, (double)b0.z, r0); r0 = fma((double)a0.w, (double)b0.w, r0);
-                    r1 = fma((double)a1.x, (double)b1.x, r1); r1 = fma((double)a1.y, (double)b1.y, r1);
-                    r1 = fma((double)a1.z, (double)b1.z, r1); r1 = fma((double)a1.w, (double)b1.w, r1);
-                    r2 = fma((double)a2.x, (double)b2.x, r2); r2 = fma((double)a2.y, (double)b2.y, r2);
-                    r2 = fma((double)a2.z, (double)b2.z, r2); r2 = fma((double)a2.w, (double)b2.w, r2);
-                    r3 = fma((double)a3.x, (double)b3.x, r3); r3 = fma((double)a3.y, (double)b3.y, r3);
-                    r3 = fma((double)a3.z, (double)b3.z, r3); r3 = fma((double)a3.w, (double)b3.w, r3);
-                }
-                for (; c < q; c += 32) {
-                    const float4 a0 = __ldg(x4 + c), b0 = __ldg(w4 + c);
-                    r0 = fma((double)a0.x, (double)b0.x, r0); r0 = fma((double)a0.y, (double)b0.y, r0);
-                    r0 = fma((double)a0.z, (double)b0.z, r0); r0 = fma((double)a0.w, (double)b0.w, r0);
-                }
-            } else {
-                int c = lane;
-                for (; c + 96 < d; c += 128) {
-                    r0 = fma((double)x[c], (double)w[c], r0);
-                    r1 = fma((double)x[c + 32], (double)w[c + 32], r1);
-                    r2 = fma((double)x[c + 64], (double)w[c + 64], r2);
-                    r3 = fma((double)x[c + 96], (double)w[c + 96], r3);
-                }
-                for (; c < d; c += 32) r0 = fma((double)x[c], (double)w[c], r0);
-            }
-            r = (r0 + r1) + (r2 + r3);
+biasreg_colsum_kernel(int d, int n_val, int rows_per_chunk, const float* __restrict__ Xv,
+                      const double* __restrict__ res, double* __restrict__ partials) {
+    pdl_trigger();
+    pdl_wait();
+    // the first sweep touched the last rows last: chunks are taken from the end, while those rows are still in L2
+    const int chunk = (int)gridDim.y - 1 - (int)blockIdx.y;
+    const int row0 = chunk * rows_per_chunk, row1 = min(n_val, row0 + rows_per_chunk);
+    double* mine = partials + (size_t)chunk * (d + 1);
+    if (VEC) {
+        const int c4 = blockIdx.x * kThreads + threadIdx.x;   // this thread's float4 of every row
+        if (c4 < (d >> 2)) {
+            const float4* col = reinterpret_cast<const float4*>(Xv) + c4;
+            const int64_t q = d >> 2;
+            double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+            int i = row0;
+            for (; i + 7 < row1; i += 8) {
+                float4 x[8];
+                double r[8];
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) r += __shfl_xor_sync(0xffffffffu, r, o);
-            r -= (double)yv[i];
-            if (lane == 0) sq += r * r;
+                for (int k = 0; k < 8; ++k) x[k] = __ldg(col + (int64_t)(i + k) * q);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) r[k] = __ldg(res + i + k);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    a0 = fma((double)x[k].x, r[k], a0); a1 = fma((double)x[k].y, r[k], a1);
+                    a2 = fma((double)x[k].z, r[k], a2); a3 = fma((double)x[k].w, r[k], a3);
+                }
+            }
+            for (; i < row1; ++i) {
+                const float4 x = __ldg(col + (int64_t)i * q);
+                const double r = __ldg(res + i);
+                a0 = fma((double)x.x, r, a0); a1 = fma((double)x.y, r, a1);
+                a2 = fma((double)x.z, r, a2); a3 = fma((double)x.w, r, a3);
+            }
+            mine[4 * c4] = a0; mine[4 * c4 + 1] = a1; mine[4 * c4 + 2] = a2; mine[4 * c4 + 3] = a3;
         }
-        if (lane == 0) r_s[warp] = (i < row1) ? r : 0.0;   // a row past the end contributes nothing
-        __syncthreads();
-        if (VEC) {
-            const int q = d >> 2;
-            for (int c = threadIdx.x; c < q; c += kThreads) {
-                float4 xv[kRows];
-#pragma unroll
-                for (int k = 0; k < kRows; ++k)
-                    xv[k] = (base + k < row1) ? __ldg(reinterpret_cast<const float4*>(Xv + (int64_t)(base + k) * d) + c)
-                                              : make_float4(0.f, 0.f, 0.f, 0.f);
-                double a0 = g_s[4 * c], a1 = g_s[4 * c + 1], a2 = g_s[4 * c + 2], a3 = g_s[4 * c + 3];
-#pragma unroll
-                for (int k = 0; k < kRows; ++k) {
-                    a0 = fma((double)xv[k].x, r_s[k], a0); a1 = fma((double)xv[k].y, r_s[k], a1);
-                    a2 = fma((double)xv[k].z, r_s[k], a2); a3 = fma((double)xv[k].w, r_s[k], a3);
-                }
-                g_s[4 * c] = a0; g_s[4 * c + 1] = a1; g_s[4 * c + 2] = a2; g_s[4 * c + 3] = a3;
-            }
-        } else {
-            for (int c = threadIdx.x; c < d; c += kThreads) {
-                float xv[kRows];
-#pragma unroll
-                for (int k = 0; k < kRows; ++k) xv[k] = (base + k < row1) ? Xv[(int64_t)(base + k) * d + c] : 0.f;
-                double a = g_s[c];
-#pragma unroll
-                for (int k = 0; k < kRows; ++k) a = fma((double)xv[k], r_s[k], a);
-                g_s[c] = a;
-            }
+    } else {
+        const int c = blockIdx.x * kThreads + threadIdx.x;
+        if (c < d) {
+            double a = 0.0;
+            for (int i = row0; i < row1; ++i) a = fma((double)Xv[(int64_t)i * d + c], __ldg(res + i), a);
+            mine[c] = a;
         }
-        __syncthreads();
     }
-    double* mine = partials + (size_t)blockIdx.x * (d + 1);
-    for (int c = threadIdx.x; c < d; c += kThreads) mine[c] = g_s[c];
-    // the block's share of the meta loss: warps in order
-    if (lane == 0) r_s[warp] = sq;
-    __syncthreads();
-    if (threadIdx.x == 0) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
         double t = 0.0;
-        for (int k = 0; k < kRows; ++k) t += r_s[k];
+        for (int i = row0; i < row1; ++i) { const double r = __ldg(res + i); t = fma(r, r, t); }
         mine[d] = t;
     }
 }
 
-// Column c of the result = 2 x (sum over blocks, in block order, of their partials); column d is the meta loss.
-__global__ void __launch_bounds__(128)
+// Column c of the result = 2 x (sum over the row chunks of their partials); column d is the meta loss.  A block
+// takes 32 columns; each of its eight warps adds a contiguous eighth of the chunks, in chunk order, and the eight
+// sums are added in warp order: a fixed order, whatever the scheduling.
+__global__ void __launch_bounds__(kThreads)
 biasreg_reduce_kernel(int d, int blocks, const double* __restrict__ partials, float* __restrict__ g_out,
                       float* __restrict__ loss_out) {
     pdl_trigger();
     pdl_wait();
-    const int c = blockIdx.x * 128 + threadIdx.x;
-    if (c > d) return;
+    __shared__ double part[kWarps][32];
+    const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
+    const int c = blockIdx.x * 32 + lane;
+    const int per = (blocks + kWarps - 1) / kWarps;
+    const int b0 = grp * per, b1 = min(blocks, b0 + per);
     double t = 0.0;
+    if (c <= d) {
 #pragma unroll 8
-    for (int b = 0; b < blocks; ++b) t += __ldcg(partials + (size_t)b * (d + 1) + c);
-    if (c < d) g_out[c] = (float)(2.0 * t);
-    else if (loss_out) *loss_out = (float)t;
+        for (int b = b0; b < b1; ++b) t += __ldcg(partials + (size_t)b * (d + 1) + c);
+    }
+    part[grp][lane] = t;
+    __syncthreads();
+    if (grp == 0 && c <= d) {
+        double sum = 0.0;
+#pragma unroll
+        for (int k = 0; k < kWarps; ++k) sum += part[k][lane];
+        if (c < d) g_out[c] = (float)(2.0 * sum);
+        else if (loss_out) *loss_out = (float)sum;
+    }
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -157,35 +211,49 @@ biasreg_fd_kernel(int64_t d, const float* __restrict__ w_plus, const float* __re
 
 }  // namespace
 
+// Row chunks of the second sweep: at least 32 rows each and no more chunks than twice the SM count (the
+// partials buffer is sized for that many).
 int biasreg_grid(const sama_ctx* ctx, int n_val) {
-    int g = (n_val + kRows - 1) / kRows;
-    if (g > 2 * ctx->sm_count) g = 2 * ctx->sm_count;
+    const int cap = 2 * ctx->sm_count;
+    int rows = (n_val + cap - 1) / cap;
+    if (rows < 32) rows = 32;
+    const int g = (n_val + rows - 1) / rows;
     return g < 1 ? 1 : g;
 }
 
+// `partials` holds biasreg_grid() x (d + 1) doubles followed by n_val doubles of residuals.
 cudaError_t launch_biasreg_direct_grad(sama_ctx* ctx, int d, int n_val, const float* Xv, const float* yv,
                                        const float* w, float* g_out, float* loss_out, cudaStream_t st) {
-    const size_t smem = sizeof(double) * ((size_t)d + kRows);
     const bool vec = (d % 4 == 0) && ((reinterpret_cast<uintptr_t>(Xv) & 15u) == 0) &&
                      ((reinterpret_cast<uintptr_t>(w) & 15u) == 0);
-    if (smem > 48 * 1024) {
-        const cudaError_t e = vec ? cudaFuncSetAttribute(biasreg_partials_kernel<true>,
-                                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-                                  : cudaFuncSetAttribute(biasreg_partials_kernel<false>,
-                                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-    }
-    const int grid = biasreg_grid(ctx, n_val);
+    const int chunks = biasreg_grid(ctx, n_val);
+    const int rows_per_chunk = (n_val + chunks - 1) / chunks;
+    double* partials = ctx->br_partials;
+    double* res = partials + (size_t)chunks * ((size_t)d + 1);
     {
+        int grid = (n_val + kWarps - 1) / kWarps;
+        if (grid > 4 * ctx->sm_count) grid = 4 * ctx->sm_count;   // one resident wave; warps stride over the rows
+        if (grid < 1) grid = 1;
         KernelScope scope(ctx, SAMA_K_BIASREG_GRAD, -1, st);
-        if (vec) biasreg_partials_kernel<true><<<grid, kThreads, smem, st>>>(d, n_val, Xv, yv, w, ctx->br_partials);
-        else biasreg_partials_kernel<false><<<grid, kThreads, smem, st>>>(d, n_val, Xv, yv, w, ctx->br_partials);
+        if (vec) biasreg_residual_kernel<true><<<grid, kThreads, 0, st>>>(d, n_val, Xv, yv, w, res);
+        else biasreg_residual_kernel<false><<<grid, kThreads, 0, st>>>(d, n_val, Xv, yv, w, res);
         const cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
+    {
+        const int strips = vec ? ((d >> 2) + kThreads - 1) / kThreads : (d + kThreads - 1) / kThreads;
+        KernelScope scope(ctx, SAMA_K_BIASREG_GRAD, -1, st);
+        const dim3 grid(strips < 1 ? 1 : strips, chunks);
+        const cudaError_t e =
+            vec ? launch_dependent(biasreg_colsum_kernel<true>, grid, dim3(kThreads), 0, st, d, n_val, rows_per_chunk, Xv,
+                                   (const double*)res, partials)
+                : launch_dependent(biasreg_colsum_kernel<false>, grid, dim3(kThreads), 0, st, d, n_val, rows_per_chunk, Xv,
+                                   (const double*)res, partials);
+        if (e != cudaSuccess) return e;
+    }
     KernelScope scope(ctx, SAMA_K_BIASREG_GRAD, -1, st);
-    return launch_dependent(biasreg_reduce_kernel, dim3((d + 1 + 127) / 128), dim3(128), 0, st, d, grid,
-                            (const double*)ctx->br_partials, g_out, loss_out);
+    return launch_dependent(biasreg_reduce_kernel, dim3((d + 1 + 31) / 32), dim3(kThreads), 0, st, d, chunks,
+                            (const double*)partials, g_out, loss_out);
 }
 
 cudaError_t launch_biasreg_fd(sama_ctx* ctx, int64_t d, const float* w_plus, const float* w_minus,

@@ -717,13 +717,14 @@ int sama_biasreg_direct_grad(sama_ctx* ctx, int32_t d, int32_t n_val, const floa
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return SAMA_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;
-    const size_t need = (size_t)biasreg_grid(ctx, n_val) * ((size_t)d + 1);
+    // the row chunks' partial gradients, then the residuals
+    const size_t need = (size_t)biasreg_grid(ctx, n_val) * ((size_t)d + 1) + (size_t)n_val;
     if (ctx->br_partials_doubles < need) {
         SAMA_CUDA(ctx, cudaStreamSynchronize(st));
         cudaFree(ctx->br_partials);
         ctx->br_partials = nullptr;
         ctx->br_partials_doubles = 0;
-        const size_t take = 2 * (size_t)ctx->sm_count * ((size_t)d + 1);
+        const size_t take = 2 * (size_t)ctx->sm_count * ((size_t)d + 1) + (size_t)n_val;
         if (cudaMalloc(&ctx->br_partials, sizeof(double) * take) != cudaSuccess) { cudaGetLastError(); return SAMA_ERR_NOMEM; }
         ctx->br_partials_doubles = take;
     }

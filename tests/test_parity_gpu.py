@@ -446,6 +446,32 @@ def test_weights_formed_in_the_operand_stage_match_the_presplit_copy(dims, batch
     assert np.isnan(poisoned["loss_plus"]).all() and np.isnan(poisoned["loss_minus"]).all()
 
 
+def test_two_contexts_keep_their_own_tensor_core_state():
+    """The tensor-core path's launch state (shared-memory opt-in, resident CTA pairs, cached tensor maps,
+    experiment switches) belongs to a context, not to the process: two contexts for different models, alive at
+    once and used alternately, give what each gives alone, and destroying one leaves the other working."""
+    cases = [W.custom_mlp((512, 2560, 40), 1280, seed=9), W.custom_mlp((40, 200, 72, 24), 257, seed=5)]
+    alone = []
+    for cfg, w in cases:
+        with Ctx(cfg.n_params, cfg.batch, cfg.dims, 2) as ctx:
+            alone.append(run_step(ctx, cfg, w, B.Adam(), 1e-2))
+    a = Ctx(cases[0][0].n_params, cases[0][0].batch, cases[0][0].dims, 2)
+    b = Ctx(cases[1][0].n_params, cases[1][0].batch, cases[1][0].dims, 2)
+    try:
+        for _ in range(2):
+            for ctx, (cfg, w), ref in ((a, cases[0], alone[0]), (b, cases[1], alone[1])):
+                got = run_step(ctx, cfg, w, B.Adam(), 1e-2)
+                assert got["status"] == 0 and B.sama_last_forward_path(ctx.h) == 2
+                for k in ("p", "metagrad", "loss_plus", "loss_minus"):
+                    assert np.array_equal(got[k], ref[k]), k
+        a.close()
+        got = run_step(b, cases[1][0], cases[1][1], B.Adam(), 1e-2)
+        assert np.array_equal(got["metagrad"], alone[1]["metagrad"]) and got["status"] == 0
+    finally:
+        a.close()
+        b.close()
+
+
 @pytest.mark.parametrize("name", ["tiny", "mlp3072"])
 def test_one_launch_sweep_against_two_launches(monkeypatch, name):
     """Small models run adaptation, norm, perturbation and operand split as ONE cooperative launch (a grid-wide
