@@ -11,7 +11,9 @@ on the 110 M / 355 M flat vectors (HBM GB/s).  ``--impl reference`` times the
 CPU checker on the host cores instead (rank 0 only).
 
 Timing: CUDA events on the launching stream around each step, an L2 flush
-(a write larger than L2) between steps outside the events, W >= 3 warm-ups,
+between steps outside the events (a write larger than L2, then a read larger
+than L2, so that the flush's own dirty lines are written back before the
+timed step instead of under its first kernel), W >= 3 warm-ups,
 barrier + synchronize on both sides, max over ranks.  ``--steps K`` is
 multiplied inside: every one of the K steps is repeated ``inner_reps`` times
 (each repetition timed by its own event pair) so that the timed region lasts
@@ -195,11 +197,11 @@ def config_for(name: str, flat_n: int = 0) -> dict:
     """The workload description both arms print (identical dicts)."""
     if name in W.FLAT_SIZES:
         return {"workload": name, "dims": None, "batch": 0, "n_params": int(flat_n or W.FLAT_SIZES[name]),
-                "alpha": 1.0, "l2": "flushed between steps (256 MiB write, outside the events)",
+                "alpha": 1.0, "l2": "flushed between steps (256 MiB written, then 256 MiB read; outside the events)",
                 "replicas": "one independent step per rank, no data-path collective"}
     cfg = W.CONFIGS[name]
     return {"workload": name, "dims": list(cfg.dims), "batch": cfg.batch, "n_params": cfg.n_params,
-            "alpha": cfg.alpha, "l2": "flushed between steps (256 MiB write, outside the events)",
+            "alpha": cfg.alpha, "l2": "flushed between steps (256 MiB written, then 256 MiB read; outside the events)",
             "replicas": "one independent step per rank, no data-path collective"}
 
 
@@ -245,8 +247,15 @@ class Bench:
         self.group = replicas.init(backend="nccl", device=self.dev)   # one process per GPU; independent replicas
         self.peaks = load_peaks()
         self.flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=self.dev)
+        self.flush_read = torch.zeros(64 * 1024 * 1024, dtype=torch.int32, device=self.dev)
         self.stream = torch.cuda.current_stream()
         self.sm_count = torch.cuda.get_device_properties(self.local).multi_processor_count
+
+    def flush(self):
+        """Cold L2 for the next step: 256 MiB written (evicts everything), then 256 MiB read (the written lines go
+        back to HBM now, not under the step's first kernel; what is left in L2 is clean)."""
+        self.flush_buf.fill_(1)
+        self.flush_read.max()
 
     def barrier(self):
         self.group.barrier()
@@ -280,8 +289,6 @@ class Bench:
         d = {k: host[k].to(dev) for k in keys}
         p, tp, tm = (torch.empty(n, dtype=torch.float32, device=dev) for _ in range(3))
         mg = torch.empty(max(B, 1), dtype=torch.float32, device=dev)
-        flush_buf = self.flush_buf
-
         outputs = {"plus": tp if args.theta_outputs == "both" else None,
                    "minus": tm if args.theta_outputs != "none" else None}
         self.store_theta_pm = args.theta_outputs == "both"
@@ -297,7 +304,7 @@ class Bench:
         def timed(K):
             ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
             for a, b in ev:
-                flush_buf.fill_(1)
+                self.flush()
                 a.record(stream)
                 one_step()
                 b.record(stream)
@@ -307,7 +314,7 @@ class Bench:
         sampler = ClockSampler(self.local)
         sampler.start()
         for _ in range(args.warmup):
-            flush_buf.fill_(1)
+            self.flush()
             one_step()
         torch.cuda.synchronize()
         # inner repetitions: enough for the timed region to last about region_s (every rank takes the same count)
@@ -447,7 +454,7 @@ class Bench:
             outputs["plus"] = None
             Kv = min(total_steps, 200)
             for _ in range(3):
-                flush_buf.fill_(1)
+                self.flush()
                 one_step()
             msv = sum(timed(Kv)) / Kv
             S.sama_profile_enable(ctx, 1)
@@ -476,7 +483,7 @@ class Bench:
             Kr = min(total_steps, 100)
             evr = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(Kr)]
             for a_, b_ in evr:
-                flush_buf.fill_(1)
+                self.flush()
                 a_.record(stream)
                 rw_step()
                 b_.record(stream)
@@ -514,7 +521,7 @@ class Bench:
             Km = max(3, min(args.steps, 50))
             evm = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(Km)]
             for a_, b_ in evm:
-                flush_buf.fill_(1)
+                self.flush()
                 a_.record(stream)
                 S.sama_meta_grad(ctx, mlp, d["theta"], d["X"], d["y"], B, gm_out, None, stream)
                 b_.record(stream)
@@ -595,7 +602,7 @@ def biased_regression_stage(b, seed):
         K = 50
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
         for a_, b_ in ev:
-            b.flush_buf.fill_(1)
+            b.flush()
             a_.record(stream)
             step()
             b_.record(stream)
