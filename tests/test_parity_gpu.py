@@ -1,7 +1,7 @@
 """GPU parity: the C-ABI CUDA path against the CPU checker, element by element,
 on the same seeded inputs.
 
-Tolerances (stated by the task this library was built for, restated here):
+Tolerances (the library's stated accuracy targets):
   adaptation / perturbation : relative 1e-5 elementwise, eps_fd relative 1e-6;
   FD meta-gradient          : |a-b| <= max(2e-3 |b|, 1e-6) elementwise, plus the
                               same 2e-3 on the whole vector in the 2-norm.
