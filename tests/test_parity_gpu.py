@@ -480,6 +480,7 @@ def test_one_launch_sweep_against_two_launches(monkeypatch, name):
     shows no expired wait.  Repeated calls of the one-launch form are bit-identical (its counters return to zero)."""
     cfg = W.CONFIGS[name]
     w = W.mlp_workload(cfg, 0)
+    monkeypatch.delenv("SAMA_NO_FUSED_SWEEP", raising=False)   # (the switch is read when a context is created)
     with Ctx(cfg.n_params, cfg.batch, cfg.dims, 2) as ctx:
         a = run_step(ctx, cfg, w, B.Adam(), 1e-2)
         a2 = run_step(ctx, cfg, w, B.Adam(), 1e-2)
