@@ -643,6 +643,8 @@ def main():
                     help="skip the extra passes on the headline workload (theta+ not stored; shared reweighting network)")
     ap.add_argument("--no-extras", action="store_true",
                     help="time only --workload (the other workloads are added by default on one GPU)")
+    ap.add_argument("--biasreg-only", action="store_true",
+                    help="run only the biased-regression stage (Appendix E) and print its record")
     ap.add_argument("--region-s", type=float, default=1.2, help="target length of the primary timed region")
     ap.add_argument("--flat-n", type=int, default=0, help="override the length of a flat-vector workload")
     ap.add_argument("--meta-grad", action="store_true",
@@ -656,6 +658,12 @@ def main():
 
     b = Bench(args)
     world, rank = b.group.world, b.group.rank
+    if args.biasreg_only:
+        rec = biased_regression_stage(b, b.group.seed)
+        if rank == 0:
+            print(json.dumps({"biased_regression": rec}), flush=True)
+        b.group.close()
+        return
     name = args.workload
     flat = name in W.FLAT_SIZES
     seed = b.group.seed  # each rank owns an independent batch / vector: no data-path collective
