@@ -143,16 +143,40 @@ softmax_grad_kernel(float* __restrict__ z, const int32_t* __restrict__ y, int B,
     }
 }
 
-// out[j] = sum_i dz[i][j], rows added in order; one thread per column.
-__global__ void __launch_bounds__(256)
+// out[j] = sum_i dz[i][j].  A block takes 32 columns; each of its 32 warps adds a contiguous share of the
+// rows in row order (sixteen loads in flight), and the warps' sums are added in warp order: a fixed order, and
+// enough rows in flight that the sweep is not a chain of B dependent loads per column.
+constexpr int kColsumWarps = 32;
+__global__ void __launch_bounds__(32 * kColsumWarps)
 colsum_kernel(const float* __restrict__ dz, int B, int N, float* __restrict__ out) {
     pdl_trigger();
     pdl_wait();
-    const int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= N) return;
+    __shared__ float part[kColsumWarps][32];
+    const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
+    const int j = blockIdx.x * 32 + lane;
+    const int per = (B + kColsumWarps - 1) / kColsumWarps;
+    const int i0 = grp * per, i1 = min(B, i0 + per);
     float s = 0.f;
-    for (int i = 0; i < B; ++i) s += dz[(int64_t)i * N + j];
-    out[j] = s;
+    if (j < N) {
+        const float* col = dz + j;
+        int i = i0;
+        for (; i + 15 < i1; i += 16) {
+            float v[16];
+#pragma unroll
+            for (int k = 0; k < 16; ++k) v[k] = col[(int64_t)(i + k) * N];
+#pragma unroll
+            for (int k = 0; k < 16; ++k) s += v[k];
+        }
+        for (; i < i1; ++i) s += col[(int64_t)i * N];
+    }
+    part[grp][lane] = s;
+    __syncthreads();
+    if (grp == 0 && j < N) {
+        float t = 0.f;
+#pragma unroll
+        for (int k = 0; k < kColsumWarps; ++k) t += part[k][lane];
+        out[j] = t;
+    }
 }
 
 // *out = (1/B) sum_i loss[i], one block, fixed order.
@@ -323,7 +347,7 @@ static cudaError_t run_meta_grad_tc(sama_ctx* ctx, const sama_mlp_t* mlp, const 
         if ((e = launch_gemm_tf32x3(ctx, tw, st)) != cudaSuccess) return e;
         {
             KernelScope scope(ctx, SAMA_K_META_AUX, l, st);
-            if ((e = launch_dependent(colsum_kernel, dim3((dout + 255) / 256), dim3(256), 0, st, dz, (int)B, dout,
+            if ((e = launch_dependent(colsum_kernel, dim3((dout + 31) / 32), dim3(32 * kColsumWarps), 0, st, dz, (int)B, dout,
                                       g_out + lay.w_off[l] + lay.w_cnt[l])) != cudaSuccess)
                 return e;
         }
@@ -419,7 +443,7 @@ static cudaError_t run_meta_grad_fma(sama_ctx* ctx, const sama_mlp_t* mlp, const
         if ((e = run_gemm(ctx, gw, l, st)) != cudaSuccess) return e;
         {
             KernelScope scope(ctx, SAMA_K_META_AUX, l, st);
-            if ((e = launch_dependent(colsum_kernel, dim3((dout + 255) / 256), dim3(256), 0, st, dz, (int)B, dout,
+            if ((e = launch_dependent(colsum_kernel, dim3((dout + 31) / 32), dim3(32 * kColsumWarps), 0, st, dz, (int)B, dout,
                                       g_out + boff[l])) != cudaSuccess)
                 return e;
         }
