@@ -33,7 +33,7 @@ def gpu_step(ctx, w, w_cur, lam, beta, alpha, adam=None, state=None):
             "metagrad": mg.cpu().numpy(), "eps_fd": read_f32(B.sama_ctx_eps_fd(ctx.h))}
 
 
-@pytest.mark.parametrize("d,n_val", [(1, 1), (5, 3), (33, 70), (256, 512), (1000, 1237), (4096, 300)])
+@pytest.mark.parametrize("d,n_val", [(1, 1), (5, 3), (33, 70), (256, 512), (1000, 1237), (4096, 300), (64, 20000)])
 @pytest.mark.parametrize("alpha", [1.0, 1e-2])
 def test_biasreg_step_parity(d, n_val, alpha):
     cfg = W.BiasRegConfig("t", d, max(2 * d, 4), n_val)
